@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the BranchGRPO tree hot path: tree node-steps/s and achieved HBM bandwidth.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one batch of synthetic trees: root init, T x
+[velocity, fused tree step], leaf rewards, reward fusion + depth-wise advantages, pruning masks.
+A node-step is one edge of a tree (one child latent with its log-prob).  With N > 1 (launched by
+torch.distributed.run) every rank runs its own shard of trees - the path has no exchange step -
+and the reported value is all ranks' node-steps over the slowest rank's time (weak scaling).
+
+`--impl reference` times the CPU oracle (oracle/), as it stands, on a bounded sample of the same
+workload on this machine's host cores; it is a deliberately slow program and a reported baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import CONFIGS, make_inputs  # noqa: E402
+
+METRIC = "tree node-steps/sec and achieved HBM GB/s (% of peak) at 1 B200 vs CPU oracle"
+UNIT = "node-steps/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM traffic per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload; reported only while the kernel source still has the
+# hash the capture was taken with.  Filled in from profiles/.
+NCU_TRAFFIC = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def kernel_source_hash(names=("tree_step.cu", "philox.cuh", "internal.h")):
+    h = hashlib.sha256()
+    for n in names:
+        h.update(open(os.path.join(ROOT, "paper_2509_06040_b200", "csrc", n), "rb").read())
+    return h.hexdigest()[:12]
+
+
+# ------------------------------------------------------------------------------------------------ algorithmic bytes
+def step_bytes_per_launch(w, n_trees):
+    """Algorithmic HBM bytes of each tree_step launch: per parent one read of z (4D) and, with a supplied
+    velocity, of v (4D); per child one write (4D); the closed-form velocity's target mean (4D per tree) is
+    read once per launch.  Node-table rows, log-probs and reduction partials are negligible and not counted."""
+    D, out, width = w.D, [], 1
+    for i in range(w.T):
+        fan = w.K if i in w.splits else 1
+        b = n_trees * width * (4 * D * (2 if w.velocity == "mlp" else 1) + fan * 4 * D)
+        if w.velocity == "linear":
+            b += n_trees * 4 * D
+        out.append(b)
+        width *= fan
+    return out
+
+
+def mlp_flops_per_launch(w, n_trees):
+    out, width = [], 1
+    for i in range(w.T):
+        out.append(n_trees * width * w.tokens * 2 * 2 * w.channels * w.hidden)
+        width *= (w.K if i in w.splits else 1)
+    return out
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 7]
+        os.unlink(self.f.name)
+        if not rows:
+            return out
+        sm = [float(r[0]) for r in rows]
+        out["sm_mhz"] = float(np.median(sm))
+        out["sm_max_mhz"] = float(rows[0][1])
+        out["power_w_max"] = max(float(r[2]) for r in rows)
+        out["samples"] = len(rows)
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for k, nm in enumerate(names):
+            if any("Active" == r[4 + k].strip() for r in rows):
+                out["reasons"].append(nm)
+        return out
+
+
+# ------------------------------------------------------------------------------------------------ oracle timing
+def oracle_pass(w, inp, sample):
+    """One pass of the oracle over a bounded sample of workload `w`.  Returns (seconds, node-steps of the
+    FULL per-GPU workload that this time corresponds to after linear scaling, description, threads)."""
+    from oracle import credit, mlp, rewards, sde
+    from oracle import tree as otree
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    sig, s0 = float(np.float32(w.sigma)), float(np.float32(w.s0))
+    t0 = time.perf_counter()
+    if w.velocity == "linear":
+        n_elem = max(4, (int(w.D * sample) // 4) * 4)
+        mu = inp.mu[0][:n_elem].astype(np.float64)
+        lat, logp = sde.rollout(topo, n_elem, grid, sig, w.branch_corr_s, w.seed,
+                                lambda z, i, p: sde.linear_velocity(z.astype(np.float64), float(grid[i]), mu, s0))
+        tgt = (inp.target if inp.target is not None else inp.mu)[0][:n_elem]
+        r = np.array([rewards.neg_mse(lat[l], tgt) for l in topo.leaf_ids()])
+        frac = n_elem / w.D
+        desc = f"1 of {w.n_trees} trees, first {n_elem} of {w.D} elements per node, all {topo.edges} node-steps; time scaled by D/sample"
+        threads = 1
+    else:
+        n_tok = max(1, int(w.tokens * sample))
+        D_s = n_tok * w.channels
+        vel = lambda z, i, p: mlp.mlp_velocity(z.reshape(n_tok, w.channels), inp.W1, inp.W2).reshape(-1)
+        lat, logp = sde.rollout(topo, D_s, grid, sig, w.branch_corr_s, w.seed, vel)
+        if inp.target is not None:
+            r = np.array([float(inp.reward_draws[0][q]) + 0.1 * rewards.cosine(lat[l], inp.target[0][:D_s])
+                          for q, l in enumerate(topo.leaf_ids())])
+        else:
+            r = inp.reward_draws[0].astype(np.float64)
+        frac = n_tok / w.tokens
+        desc = f"1 of {w.n_trees} trees, first {n_tok} of {w.tokens} tokens per node, all {topo.edges} node-steps; time scaled by tokens/sample"
+        threads = _blas_threads()
+    rbar = credit.fuse_rewards(topo, r, logp, w.beta)
+    credit.depth_advantages(topo, rbar, float(np.float32(w.eps)))
+    credit.gradient_mask(topo, rbar.astype(np.float32), w.width_mode, w.width_k, inp.pruned_steps, w.ignore_last_step)
+    dt = time.perf_counter() - t0
+    full_seconds_one_tree = dt / frac
+    return dt, topo.edges / full_seconds_one_tree, desc, threads
+
+
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample_fraction(w):
+    return {"toy": 1.0, "image": 0.05, "image_batch": 0.05, "group": 0.01, "video": 0.25}.get(w.name, 0.05)
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = make_inputs(w.scaled(n_trees=1))
+    frac = oracle_sample_fraction(w)
+    for _ in range(args.warmup):
+        oracle_pass(w, inp, frac / 8)
+    vals, secs = [], []
+    for _ in range(args.steps):
+        dt, v, desc, threads = oracle_pass(w, inp, frac)
+        vals.append(v)
+        secs.append(dt)
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * w.n_trees * w.node_steps / value, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "description": w.description, "n_trees": w.n_trees,
+                   "note": "CPU oracle on host cores; ms_per_step is the full batch extrapolated from the sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+                         "sample_seconds": float(np.mean(secs))},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import __graft_entry__
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2509_06040_b200.session import TreeSession
+    from paper_2509_06040_b200 import binding as B
+
+    # weak scaling: every rank holds the workload's n_trees trees, with its own global tree indices
+    base = rank * w.n_trees
+    inp = make_inputs(w, tree_base=base)
+    s = TreeSession(w, tree_id_base=base, device=f"cuda:{local}")
+    s.upload_inputs(inp)
+    pool_bytes = s.latents.numel() * 4
+    flush = pool_bytes <= 2 * L2_BYTES
+    flush_buf = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=s.device) if flush else None
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for k in range(args.warmup):
+        s.run_all(seed=w.seed + k)
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+
+    # ---- timed region: K passes, device-timed with CUDA events on the launching stream
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    sync_all()
+    for k in range(args.steps):
+        if flush:
+            flush_buf.fill_(float(k))
+        ev[k][0].record()
+        s.run_all(seed=w.seed + 1000 + k)
+        ev[k][1].record()
+    sync_all()
+    clocks = sampler.stop() if sampler else None
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    t = torch.tensor([total_ms], dtype=torch.float64, device=s.device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    node_steps_per_pass = world * w.n_trees * w.node_steps
+    value = node_steps_per_pass * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the C ABI with host buffers: H2D of the step's inputs (pinned), D2H of its results
+    host_in = {}
+    for name in ("mu", "target", "reward_draws"):
+        a = getattr(inp, name)
+        if a is not None:
+            host_in[name] = torch.from_numpy(a).pin_memory()
+    host_out = {n: torch.empty_like(getattr(s, n), device="cpu").pin_memory() for n in ("adv", "mask", "logp", "leaf_r")}
+    h2d = sum(x.numel() * x.element_size() for x in host_in.values())
+    d2h = sum(x.numel() * x.element_size() for x in host_out.values())
+
+    def e2e_pass(k):
+        for name, h in host_in.items():
+            getattr(s, name).copy_(h, non_blocking=True)
+        s.run_all(seed=w.seed + 2000 + k)
+        for name, h in host_out.items():
+            h.copy_(getattr(s, name), non_blocking=True)
+
+    for k in range(2):
+        e2e_pass(k)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_e2e = max(3, args.steps // 2)
+    e2e_ms = 0.0
+    for k in range(n_e2e):
+        if flush:
+            flush_buf.fill_(float(k))
+        e0.record()
+        e2e_pass(k)
+        e1.record()
+        e1.synchronize()
+        e2e_ms += e0.elapsed_time(e1)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device=s.device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = node_steps_per_pass * n_e2e / (float(t.item()) * 1e-3)
+
+    # ---- per-kernel durations, measured live with events around each launch (rank 0)
+    roof = roof_step = None
+    breakdown = {}
+    if rank == 0:
+        peaks = load_peaks()
+        reps = max(3, min(10, args.steps))
+        t_step = np.zeros(w.T)
+        t_mlp = np.zeros(w.T)
+        t_other = 0.0
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        for rep in range(reps):
+            if flush:
+                flush_buf.fill_(1.0)
+            a.record()
+            s.init(seed=w.seed + 3000 + rep)
+            b.record()
+            b.synchronize()
+            t_other += a.elapsed_time(b)
+            for i in range(w.T):
+                a.record()
+                if w.velocity == "mlp":
+                    B.velocity_mlp(s.tree, s.packed, w.hidden, s.v)
+                b.record()
+                B.tree_step(s.tree, 1 if i in w.splits else 0, s.v if w.velocity == "mlp" else None)
+                c.record()
+                c.synchronize()
+                t_mlp[i] += a.elapsed_time(b)
+                t_step[i] += b.elapsed_time(c)
+            a.record()
+            s.rewards()
+            s.fuse_advantage()
+            s.prune()
+            b.record()
+            b.synchronize()
+            t_other += a.elapsed_time(b)
+        t_step /= reps
+        t_mlp /= reps
+        t_other /= reps
+        sb = np.array(step_bytes_per_launch(w, w.n_trees), dtype=np.float64)
+        step_gbs = sb.sum() / (t_step.sum() * 1e-3) / 1e9
+        widest = int(np.argmax(sb))
+        hbm_peak = float(peaks["hbm_gbs"])
+        roof_step = {"bound": "hbm", "kernel": "step_kernel", "achieved": step_gbs, "peak": hbm_peak, "unit": "GB/s",
+                     "frac": step_gbs / hbm_peak, "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                     "peak_source": peaks["_source"], "launches_per_pass": w.T,
+                     "bytes_per_pass": float(sb.sum()), "ms_per_pass": float(t_step.sum()),
+                     "widest_launch": {"step": widest, "bytes": float(sb[widest]), "ms": float(t_step[widest]),
+                                       "gbs": float(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
+                     "traffic": None}
+        tr = NCU_TRAFFIC.get(w.name)
+        if tr and tr.get("source_hash") == kernel_source_hash():
+            roof_step["traffic"] = tr["bytes_per_launch"]
+        breakdown = {"step_ms": float(t_step.sum()), "mlp_ms": float(t_mlp.sum()), "other_ms": float(t_other)}
+        if w.velocity == "mlp" and t_mlp.sum() > t_step.sum():
+            fl = np.array(mlp_flops_per_launch(w, w.n_trees), dtype=np.float64)
+            tf = fl.sum() / (t_mlp.sum() * 1e-3) / 1e12
+            peak_tf = float(peaks["bf16_tflops"])
+            roof = {"bound": "tensor", "kernel": "mlp_velocity_kernel", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": tf / peak_tf, "peak_source": peaks["_source"], "launches_per_pass": w.T,
+                    "flops_per_pass": float(fl.sum()), "ms_per_pass": float(t_mlp.sum()), "traffic": None}
+        else:
+            roof = roof_step
+
+    # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        inp1 = make_inputs(w.scaled(n_trees=1))
+        dt, v, desc, threads = oracle_pass(w, inp1, oracle_sample_fraction(w))
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "sample_seconds": dt}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.velocity == "linear" else "f32 (step) + bf16/f32-accumulate (MLP velocity)",
+            "data": "synthetic",
+            "config": {"workload": w.name, "description": w.description, "n_trees_per_gpu": w.n_trees,
+                       "tokens": w.tokens, "channels": w.channels, "T": w.T, "K": w.K, "splits": list(w.splits),
+                       "node_steps_per_tree": w.node_steps, "model_evals_per_tree": w.model_evals,
+                       "model_evals_sequential": w.leaves * w.T, "latent_pool_bytes": pool_bytes,
+                       "l2": "flushed between steps (pool fits in L2)" if flush else "latent pool larger than L2",
+                       "parallelism": f"dp{world} over trees, no collective"},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": s.kernel_launches_per_pass() * args.steps,
+            "clocks": clocks, "kernel_ms_per_pass": breakdown,
+        }
+        if roof is not roof_step:
+            line["roofline_step"] = roof_step
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="video", choices=list(CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = CONFIGS[args.workload]
+    if args.impl == "reference":
+        args.steps = min(args.steps, 5)
+        args.warmup = min(args.warmup, 1)
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

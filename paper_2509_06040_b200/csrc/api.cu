@@ -1,0 +1,460 @@
+// C ABI of the library: argument checks, the host mirror of the tree layout, per-step coefficients and launches.
+// No device memory is allocated here; every kernel is enqueued on the caller's stream.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace bgrpo;
+
+namespace {
+
+thread_local char g_last_error[256] = "";
+
+bgrpo_status cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+    return BGRPO_ERR_CUDA;
+}
+bgrpo_status fail(bgrpo_status s, const char* why) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s", why);
+    return s;
+}
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bgrpo_status check_desc(const bgrpo_tree_desc* d) {
+    if (!d) return fail(BGRPO_ERR_INVALID_ARG, "desc is NULL");
+    if (d->n_trees < 1 || d->tokens < 1 || d->channels < 1) return fail(BGRPO_ERR_INVALID_ARG, "n_trees, tokens, channels must be >= 1");
+    const int64_t D = static_cast<int64_t>(d->tokens) * d->channels;
+    if (D % 4 != 0) return fail(BGRPO_ERR_INVALID_ARG, "tokens*channels must be a multiple of 4");
+    if (D / 4 > 0x7fffffffLL) return fail(BGRPO_ERR_INVALID_ARG, "row too long for the 32-bit block counter");
+    if (d->T < 1 || d->T > BGRPO_MAX_T) return fail(BGRPO_ERR_INVALID_ARG, "T out of range");
+    if (d->K < 1 || d->K > BGRPO_MAX_K) return fail(BGRPO_ERR_INVALID_ARG, "K out of range");
+    if (d->nodes_cap < d->T + 1) return fail(BGRPO_ERR_INVALID_ARG, "nodes_cap smaller than a split-free tree");
+    if (d->tree_id_base < 0) return fail(BGRPO_ERR_INVALID_ARG, "tree_id_base negative");
+    if (!(d->sigma >= 0.0f) || !std::isfinite(d->sigma)) return fail(BGRPO_ERR_INVALID_ARG, "sigma must be finite and >= 0");
+    if (std::isnan(d->branch_corr_s)) return fail(BGRPO_ERR_INVALID_ARG, "branch_corr_s is NaN");
+    return BGRPO_OK;
+}
+
+int nchunks_of(int64_t D) { return static_cast<int>((D / 4 + kChunkVec - 1) / kChunkVec); }
+
+size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
+    const int64_t rows = static_cast<int64_t>(d->n_trees) * d->nodes_cap;
+    const int64_t D = static_cast<int64_t>(d->tokens) * d->channels;
+    size_t b = kScratchHeader;
+    b += ((static_cast<size_t>(rows) * sizeof(unsigned int) + 255) / 256) * 256;
+    b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
+    return b;
+}
+
+void fill_coefficients(bgrpo_tree* t) {
+    const double sigma = t->desc.sigma;
+    for (int i = 0; i < t->desc.T; ++i) {
+        const double ti = t->t_grid[i], h = static_cast<double>(t->t_grid[i]) - static_cast<double>(t->t_grid[i + 1]);
+        const double c = sigma * sigma * h / (2.0 * ti);
+        const double a = 1.0 - c, b = -(h + c * (1.0 - ti));
+        StepCoef& k = t->coef[i];
+        k.a = static_cast<float>(a);
+        k.b = static_cast<float>(b);
+        const double g = sigma * std::sqrt(h);
+        k.g = static_cast<float>(g);
+        k.inv_2g2 = g > 0 ? static_cast<float>(1.0 / (2.0 * g * g)) : 0.0f;
+        k.logp_const = g > 0 ? static_cast<float>(-std::log(g) - 0.5 * std::log(2.0 * M_PI)) : 0.0f;
+        if (t->mu) {
+            const double s0 = t->s0;
+            const double ct = (1.0 - ti) * (1.0 - ti) * s0 * s0 + ti * ti;
+            const double kt = (ti - (1.0 - ti) * s0 * s0) / ct;
+            // v = kt z - (1 + kt (1-t)) mu  =>  mean = (a + b kt) z - b (1 + kt (1-t)) mu
+            k.lin_a = static_cast<float>(a + b * kt);
+            k.lin_b = static_cast<float>(-b * (1.0 + kt * (1.0 - ti)));
+        } else {
+            k.lin_a = k.lin_b = 0.0f;
+        }
+    }
+}
+
+bool tree_complete(const bgrpo_tree* t) { return t->depth == t->desc.T; }
+
+}  // namespace
+
+extern "C" {
+
+const char* bgrpo_status_string(bgrpo_status s) {
+    switch (s) {
+        case BGRPO_OK: return "ok";
+        case BGRPO_ERR_INVALID_ARG: return "invalid argument";
+        case BGRPO_ERR_STATE: return "call out of order for the tree's state";
+        case BGRPO_ERR_CAPACITY: return "capacity exceeded";
+        case BGRPO_ERR_NONFINITE: return "non-finite value met on the device";
+        case BGRPO_ERR_CUDA: return "CUDA error";
+        case BGRPO_ERR_UNSUPPORTED: return "unsupported";
+    }
+    return "unknown status";
+}
+
+const char* bgrpo_last_error(void) { return g_last_error; }
+
+bgrpo_status bgrpo_tree_workspace(const bgrpo_tree_desc* desc, bgrpo_sizes* out) {
+    if (!out) return fail(BGRPO_ERR_INVALID_ARG, "out is NULL");
+    bgrpo_status st = check_desc(desc);
+    if (st != BGRPO_OK) return st;
+    const size_t rows = static_cast<size_t>(desc->n_trees) * desc->nodes_cap;
+    const size_t D = static_cast<size_t>(desc->tokens) * desc->channels;
+    out->latents_bytes = rows * D * sizeof(float);
+    out->node_table_bytes = 4 * rows * sizeof(int32_t);
+    out->per_node_float_bytes = rows * sizeof(float);
+    out->mask_bytes = rows;
+    out->scratch_bytes = scratch_bytes_of(desc);
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_count(int32_t T, int32_t K, const int32_t* split_steps, int32_t n_splits, int64_t* nodes,
+                              int64_t* node_steps, int64_t* model_evals, int64_t* leaves) {
+    if (T < 1 || T > BGRPO_MAX_T || K < 1 || K > BGRPO_MAX_K || n_splits < 0 || n_splits > T || (n_splits > 0 && !split_steps))
+        return fail(BGRPO_ERR_INVALID_ARG, "bad schedule");
+    bool is_split[BGRPO_MAX_T] = {false};
+    for (int q = 0; q < n_splits; ++q) {
+        if (split_steps[q] < 0 || split_steps[q] >= T || is_split[split_steps[q]]) return fail(BGRPO_ERR_INVALID_ARG, "split steps must be distinct and in 0..T-1");
+        is_split[split_steps[q]] = true;
+    }
+    int64_t w = 1, total = 1;
+    for (int i = 0; i < T; ++i) {
+        if (is_split[i]) w *= K;
+        if (w > (1LL << 40)) return fail(BGRPO_ERR_CAPACITY, "tree too wide");
+        total += w;
+    }
+    if (nodes) *nodes = total;
+    if (node_steps) *node_steps = total - 1;
+    if (model_evals) *model_evals = total - w;
+    if (leaves) *leaves = w;
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b, void* stream, bgrpo_tree** out) {
+    if (!out) return fail(BGRPO_ERR_INVALID_ARG, "out is NULL");
+    bgrpo_status st = check_desc(desc);
+    if (st != BGRPO_OK) return st;
+    if (!b || !b->latents || !b->node_table || !b->logp || !b->rbar || !b->adv || !b->mask || !b->scratch)
+        return fail(BGRPO_ERR_INVALID_ARG, "a device buffer is NULL");
+    if (!desc->t_grid) return fail(BGRPO_ERR_INVALID_ARG, "t_grid is NULL");
+    if (!aligned(b->latents, 16) || !aligned(b->scratch, 256) || !aligned(b->node_table, 4) || !aligned(b->logp, 4))
+        return fail(BGRPO_ERR_INVALID_ARG, "misaligned device buffer");
+    for (int i = 0; i <= desc->T; ++i) {
+        const float t = desc->t_grid[i];
+        if (!std::isfinite(t) || t > 1.0f || t < 0.0f) return fail(BGRPO_ERR_INVALID_ARG, "t_grid values must lie in [0, 1]");
+        if (i > 0 && !(t < desc->t_grid[i - 1])) return fail(BGRPO_ERR_INVALID_ARG, "t_grid must be strictly decreasing");
+    }
+    if (!(desc->t_grid[desc->T - 1] > 0.0f)) return fail(BGRPO_ERR_INVALID_ARG, "t_grid[T-1] must be > 0");
+    if (b->scratch_bytes < scratch_bytes_of(desc)) return fail(BGRPO_ERR_CAPACITY, "scratch_bytes too small");
+    const int64_t last_id = (desc->tree_id_base + desc->n_trees) * static_cast<int64_t>(desc->nodes_cap);
+    if (last_id > 0xffffffffLL) return fail(BGRPO_ERR_CAPACITY, "global node ids exceed 32 bits");
+
+    bgrpo_tree* t = new (std::nothrow) bgrpo_tree();
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "out of host memory");
+    t->desc = *desc;
+    t->buf = *b;
+    std::memcpy(t->t_grid, desc->t_grid, sizeof(float) * (desc->T + 1));
+    t->desc.t_grid = t->t_grid;
+    t->D = static_cast<int64_t>(desc->tokens) * desc->channels;
+    t->nchunks = nchunks_of(t->D);
+    t->independent = !(std::isfinite(desc->branch_corr_s) && desc->branch_corr_s >= 0.0f);
+    if (t->independent) {
+        t->mix_shared = 0.0f;
+        t->mix_innov = 1.0f;
+    } else {
+        const double s = desc->branch_corr_s, n = std::sqrt(1.0 + s * s);
+        t->mix_shared = static_cast<float>(1.0 / n);
+        t->mix_innov = static_cast<float>(s / n);
+    }
+    t->mu = nullptr;
+    t->s0 = 0.0f;
+    char* sc = static_cast<char*>(b->scratch);
+    const size_t rows = static_cast<size_t>(desc->n_trees) * desc->nodes_cap;
+    t->status = reinterpret_cast<int32_t*>(sc);
+    t->counters = reinterpret_cast<unsigned int*>(sc + kScratchHeader);
+    t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
+    fill_coefficients(t);
+    st = bgrpo_tree_reset(t, desc->seed, stream);
+    if (st != BGRPO_OK) {
+        delete t;
+        return st;
+    }
+    *out = t;
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_reset(bgrpo_tree* t, uint64_t seed, void* stream) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    t->desc.seed = seed;
+    t->depth = 0;
+    std::memset(&t->lv, 0, sizeof(t->lv));
+    t->lv.width[0] = 1;
+    t->lv.offset[0] = 0;
+    t->lv.offset[1] = 1;
+    cudaError_t e = launch_root(t, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "root kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* t, const float* mu_dev, float s0) {
+    if (!t || !mu_dev) return fail(BGRPO_ERR_INVALID_ARG, "tree or mu is NULL");
+    if (!(s0 > 0.0f) || !std::isfinite(s0)) return fail(BGRPO_ERR_INVALID_ARG, "s0 must be finite and > 0");
+    if (!aligned(mu_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "mu misaligned");
+    t->mu = mu_dev;
+    t->s0 = s0;
+    fill_coefficients(t);
+    return BGRPO_OK;
+}
+
+static void fill_step_launch(const bgrpo_tree* t, int step, const float* v_dev, StepLaunch* p) {
+    const StepCoef& k = t->coef[step];
+    p->latents = t->buf.latents;
+    p->v = v_dev;
+    p->mu = v_dev ? nullptr : t->mu;
+    p->logp = t->buf.logp;
+    p->table = t->buf.node_table;
+    p->partials = t->partials;
+    p->counters = t->counters;
+    p->D = t->D;
+    p->n_trees = t->desc.n_trees;
+    p->nodes_cap = t->desc.nodes_cap;
+    p->nchunks = t->nchunks;
+    p->step = step;
+    p->node_id_base = static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap);
+    p->key0 = static_cast<uint32_t>(t->desc.seed);
+    p->key1 = static_cast<uint32_t>(t->desc.seed >> 32);
+    p->ca = v_dev ? k.a : k.lin_a;
+    p->cb = v_dev ? k.b : k.lin_b;
+    p->g = k.g;
+    p->inv_2g2 = k.inv_2g2;
+    p->logp_const = k.logp_const;
+    p->mix_shared = t->mix_shared;
+    p->mix_innov = t->mix_innov;
+}
+
+bgrpo_status bgrpo_tree_step(bgrpo_tree* t, int32_t split_flag, const float* v_dev, void* stream) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    if (t->depth >= t->desc.T) return fail(BGRPO_ERR_STATE, "tree already at depth T");
+    if (!v_dev && !t->mu) return fail(BGRPO_ERR_STATE, "no velocity: pass v_dev or bind a linear velocity");
+    if (v_dev && !aligned(v_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "v misaligned");
+    const int i = t->depth;
+    const int fan = split_flag ? t->desc.K : 1;
+    const int64_t W_out = static_cast<int64_t>(t->lv.width[i]) * fan;
+    const int64_t off_out = t->lv.offset[i + 1];
+    if (off_out + W_out > t->desc.nodes_cap) return fail(BGRPO_ERR_CAPACITY, "children exceed nodes_cap");
+    StepLaunch p;
+    fill_step_launch(t, i, v_dev, &p);
+    p.W_in = t->lv.width[i];
+    p.off_in = t->lv.offset[i];
+    p.off_out = static_cast<int32_t>(off_out);
+    p.fan = fan;
+    p.is_split = split_flag ? 1 : 0;
+    p.shared_noise = (split_flag && !t->independent && t->coef[i].g > 0.0f) ? 1 : 0;
+    p.write_children = 1;
+    p.logp_out = t->buf.logp;
+    cudaError_t e = launch_step(p, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "step kernel");
+    t->lv.fanout[i] = fan;
+    t->lv.width[i + 1] = static_cast<int32_t>(W_out);
+    t->lv.offset[i + 2] = static_cast<int32_t>(off_out + W_out);
+    t->depth = i + 1;
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_logprob(bgrpo_tree* t, int32_t step, const float* v_dev, float* logp_out_dev, void* stream) {
+    if (!t || !logp_out_dev) return fail(BGRPO_ERR_INVALID_ARG, "tree or output is NULL");
+    if (step < -1 || step >= t->depth) return fail(BGRPO_ERR_STATE, "step has not been taken");
+    if (step == -1 && v_dev) return fail(BGRPO_ERR_INVALID_ARG, "step -1 works with the bound linear velocity only");
+    if (!v_dev && !t->mu) return fail(BGRPO_ERR_STATE, "no velocity: pass v_dev or bind a linear velocity");
+    if (v_dev && !aligned(v_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "v misaligned");
+    const int first = step < 0 ? 0 : step, last = step < 0 ? t->depth - 1 : step;
+    for (int i = first; i <= last; ++i) {
+        StepLaunch p;
+        fill_step_launch(t, i, v_dev, &p);
+        p.W_in = t->lv.width[i];
+        p.off_in = t->lv.offset[i];
+        p.off_out = t->lv.offset[i + 1];
+        p.fan = t->lv.fanout[i];
+        p.is_split = 0;
+        p.shared_noise = 0;
+        p.write_children = 0;
+        p.logp_out = logp_out_dev;
+        cudaError_t e = launch_step(p, as_stream(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "logprob kernel");
+    }
+    return BGRPO_OK;
+}
+
+static bgrpo_status reward_common(bgrpo_tree* t, const float* target, float scale, float* r, int mode, void* stream) {
+    if (!t || !target || !r) return fail(BGRPO_ERR_INVALID_ARG, "tree, target or output is NULL");
+    if (!tree_complete(t)) return fail(BGRPO_ERR_STATE, "tree is not complete");
+    if (!aligned(target, 16)) return fail(BGRPO_ERR_INVALID_ARG, "target misaligned");
+    RewardLaunch p;
+    p.latents = t->buf.latents;
+    p.target = target;
+    p.r = r;
+    p.partials = t->partials;
+    p.counters = t->counters;
+    p.D = t->D;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.nchunks = t->nchunks;
+    p.leaves = t->lv.width[t->desc.T];
+    p.off_leaf = t->lv.offset[t->desc.T];
+    p.scale = scale;
+    p.mode = mode;
+    cudaError_t e = launch_reward(p, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "reward kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_leaf_reward_mse(bgrpo_tree* t, const float* target_dev, float* r_out_dev, void* stream) {
+    return reward_common(t, target_dev, 0.0f, r_out_dev, 0, stream);
+}
+bgrpo_status bgrpo_leaf_reward_cos(bgrpo_tree* t, const float* target_dev, float scale, float* r_inout_dev, void* stream) {
+    return reward_common(t, target_dev, scale, r_inout_dev, 1, stream);
+}
+
+bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* t, const float* leaf_rewards_dev, float beta, float logp_scale,
+                                       float eps, float adv_clip_max, void* stream) {
+    if (!t || !leaf_rewards_dev) return fail(BGRPO_ERR_INVALID_ARG, "tree or rewards is NULL");
+    if (!tree_complete(t)) return fail(BGRPO_ERR_STATE, "tree is not complete");
+    if (!std::isfinite(beta) || !std::isfinite(logp_scale) || !(eps >= 0.0f) || std::isnan(adv_clip_max))
+        return fail(BGRPO_ERR_INVALID_ARG, "beta, logp_scale must be finite and eps >= 0");
+    FuseLaunch p;
+    p.leaf_r = leaf_rewards_dev;
+    p.logp = t->buf.logp;
+    p.rbar = t->buf.rbar;
+    p.adv = t->buf.adv;
+    p.status = t->status;
+    p.lv = t->lv;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.T = t->desc.T;
+    p.nodes = t->lv.offset[t->desc.T + 1];
+    p.beta_scaled = static_cast<double>(beta) * static_cast<double>(logp_scale);
+    p.eps = eps;
+    p.clip = adv_clip_max;
+    if (static_cast<size_t>(p.nodes) * 16 > 200 * 1024) return fail(BGRPO_ERR_UNSUPPORTED, "tree too large for one CTA's shared memory");
+    cudaError_t e = launch_fuse_advantage(p, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "fuse kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_prune(bgrpo_tree* t, int32_t width_mode, int32_t k_or_b, const int32_t* pruned_steps_host,
+                              int32_t n_pruned, int32_t ignore_last_step, void* stream) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    if (!tree_complete(t)) return fail(BGRPO_ERR_STATE, "tree is not complete");
+    if (width_mode < BGRPO_WIDTH_NONE || width_mode > BGRPO_WIDTH_EXTREME_B) return fail(BGRPO_ERR_INVALID_ARG, "unknown width mode");
+    if (width_mode != BGRPO_WIDTH_NONE && k_or_b < 1) return fail(BGRPO_ERR_INVALID_ARG, "k_or_b must be >= 1");
+    if (n_pruned < 0 || (n_pruned > 0 && !pruned_steps_host)) return fail(BGRPO_ERR_INVALID_ARG, "bad pruned_steps");
+    PruneLaunch p;
+    p.pruned_bits = 0;
+    for (int q = 0; q < n_pruned; ++q) {
+        if (pruned_steps_host[q] < 0 || pruned_steps_host[q] >= t->desc.T) return fail(BGRPO_ERR_INVALID_ARG, "pruned step out of range");
+        p.pruned_bits |= 1ull << pruned_steps_host[q];
+    }
+    p.rbar = t->buf.rbar;
+    p.table = t->buf.node_table;
+    p.mask = t->buf.mask;
+    p.lv = t->lv;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.T = t->desc.T;
+    p.nodes = t->lv.offset[t->desc.T + 1];
+    p.mode = width_mode;
+    p.k = k_or_b;
+    p.last_split = -1;
+    for (int i = 0; i < t->desc.T; ++i)
+        if (t->lv.fanout[i] > 1) p.last_split = i;
+    p.ignore_last = ignore_last_step ? 1 : 0;
+    if (static_cast<size_t>(p.nodes) > 200 * 1024) return fail(BGRPO_ERR_UNSUPPORTED, "tree too large for one CTA's shared memory");
+    cudaError_t e = launch_prune(p, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "prune kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_depth_window(int32_t iter, int32_t start, int32_t size, int32_t every, int32_t stop, int32_t* steps_out, int32_t* n_out) {
+    if (!steps_out || !n_out || iter < 0 || start < 0 || size < 1 || every < 1) return fail(BGRPO_ERR_INVALID_ARG, "bad window arguments");
+    if (stop >= 0 && stop - size < 0) return fail(BGRPO_ERR_INVALID_ARG, "stop leaves no room for the window");
+    int first = start + iter / every;
+    if (stop >= 0 && first > stop - size) first = stop - size;
+    for (int j = 0; j < size; ++j) steps_out[j] = first + j;
+    *n_out = size;
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_stats(const bgrpo_tree* t, int32_t* depth, int64_t* nodes, int64_t* node_steps, int64_t* model_evals, int64_t* frontier_width) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    const int64_t n = t->lv.offset[t->depth + 1];
+    if (depth) *depth = t->depth;
+    if (nodes) *nodes = n;
+    if (node_steps) *node_steps = n - 1;
+    if (model_evals) *model_evals = t->lv.offset[t->depth];      // every node above the frontier was evaluated once
+    if (frontier_width) *frontier_width = t->lv.width[t->depth];
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_levels(const bgrpo_tree* t, int32_t n, int32_t* widths_out, int32_t* offsets_out) {
+    if (!t || n < 0 || !widths_out || !offsets_out) return fail(BGRPO_ERR_INVALID_ARG, "bad arguments");
+    for (int d = 0; d <= t->depth && d < n; ++d) {
+        widths_out[d] = t->lv.width[d];
+        offsets_out[d] = t->lv.offset[d];
+    }
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* t, void* stream) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, t->status, sizeof(word), cudaMemcpyDeviceToHost, as_stream(stream));
+    if (e == cudaSuccess) e = cudaMemsetAsync(t->status, 0, sizeof(word), as_stream(stream));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "status read");
+    return (word & 1) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
+}
+
+bgrpo_status bgrpo_philox_words_fill(uint64_t seed, uint32_t node_id, uint32_t step, uint32_t tag, uint32_t* out_dev, int64_t n_blocks, void* stream) {
+    if (!out_dev || n_blocks < 0 || !aligned(out_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "bad output");
+    cudaError_t e = launch_philox_words(seed, node_id, step, tag, out_dev, n_blocks, as_stream(stream));
+    return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "philox words kernel");
+}
+bgrpo_status bgrpo_philox_normal_fill(uint64_t seed, uint32_t node_id, uint32_t step, uint32_t tag, float* out_dev, int64_t n, void* stream) {
+    if (!out_dev || n < 0 || n % 4 != 0 || !aligned(out_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "bad output or n % 4 != 0");
+    cudaError_t e = launch_philox_normals(seed, node_id, step, tag, out_dev, n, as_stream(stream));
+    return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "philox normals kernel");
+}
+
+size_t bgrpo_velocity_mlp_packed_bytes(int32_t hidden) {
+    if (hidden < BGRPO_MLP_HIDDEN_MULTIPLE || hidden % BGRPO_MLP_HIDDEN_MULTIPLE != 0) return 0;
+    return mlp_packed_bytes(hidden);
+}
+
+bgrpo_status bgrpo_velocity_mlp_pack(const uint16_t* W1, const uint16_t* W2, int32_t hidden, void* packed_dev, void* stream) {
+    if (!W1 || !W2 || !packed_dev) return fail(BGRPO_ERR_INVALID_ARG, "NULL pointer");
+    if (hidden < BGRPO_MLP_HIDDEN_MULTIPLE || hidden % BGRPO_MLP_HIDDEN_MULTIPLE != 0) return fail(BGRPO_ERR_INVALID_ARG, "hidden must be a positive multiple of 128");
+    if (!aligned(packed_dev, 1024)) return fail(BGRPO_ERR_INVALID_ARG, "packed buffer must be 1024-byte aligned");
+    cudaError_t e = launch_mlp_pack(W1, W2, hidden, packed_dev, as_stream(stream));
+    return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp pack kernel");
+}
+
+bgrpo_status bgrpo_velocity_mlp(bgrpo_tree* t, const void* packed_dev, int32_t hidden, float* v_out_dev, void* stream) {
+    if (!t || !packed_dev || !v_out_dev) return fail(BGRPO_ERR_INVALID_ARG, "NULL pointer");
+    if (t->desc.channels != BGRPO_MLP_CHANNELS) return fail(BGRPO_ERR_UNSUPPORTED, "the MLP stage needs 64 channels");
+    if (hidden < BGRPO_MLP_HIDDEN_MULTIPLE || hidden % BGRPO_MLP_HIDDEN_MULTIPLE != 0) return fail(BGRPO_ERR_INVALID_ARG, "hidden must be a positive multiple of 128");
+    if (!aligned(packed_dev, 1024) || !aligned(v_out_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "misaligned buffer");
+    if (t->depth >= t->desc.T) return fail(BGRPO_ERR_STATE, "tree already at depth T");
+    const int i = t->depth;
+    cudaError_t e = launch_mlp(t->buf.latents, static_cast<int64_t>(t->desc.nodes_cap) * t->D, static_cast<int64_t>(t->lv.offset[i]) * t->D,
+                               t->desc.n_trees, static_cast<int64_t>(t->lv.width[i]) * t->desc.tokens, packed_dev, hidden,
+                               v_out_dev, as_stream(stream));
+    return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp kernel");
+}
+
+void bgrpo_tree_destroy(bgrpo_tree* t) { delete t; }
+
+}  // extern "C"

@@ -1,0 +1,107 @@
+// Host-side state of a batch of rollout trees and the launch interfaces of the kernels.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/bgrpo.h"
+
+namespace bgrpo {
+
+constexpr int kChunkVec = 1024;        // float4 per (parent, chunk) work item of the streaming kernels
+constexpr int kStreamThreads = 256;    // threads per CTA of the streaming kernels
+constexpr int kScratchHeader = 256;    // bytes reserved at the start of scratch for the status word
+
+// Per-step scalars of the Euler-Maruyama mean and the Gaussian transition, computed in double on the host.
+//   mean = a*z + b*v                       (v given)
+//        = lin_a*z + lin_b*mu              (closed-form velocity v = k z - (1 + k(1-t)) mu folded in)
+struct StepCoef {
+    float a, b;          // a = 1 - c, b = -(h + c (1-t)), c = sigma^2 h / (2 t)
+    float lin_a, lin_b;  // valid once a linear velocity is bound
+    float g;             // sigma sqrt(h)
+    float inv_2g2;       // 1 / (2 g^2), 0 when g == 0
+    float logp_const;    // -ln g - 0.5 ln(2 pi), 0 when g == 0
+};
+
+struct LevelInfo {                       // layout of the tree grown so far
+    int32_t width[BGRPO_MAX_T + 1];
+    int32_t offset[BGRPO_MAX_T + 2];
+    int32_t fanout[BGRPO_MAX_T];         // children per node produced by step i (K or 1)
+};
+
+}  // namespace bgrpo
+
+struct bgrpo_tree {
+    bgrpo_tree_desc desc;
+    bgrpo_buffers buf;
+    float t_grid[BGRPO_MAX_T + 1];
+    bgrpo::StepCoef coef[BGRPO_MAX_T];
+    bgrpo::LevelInfo lv;
+    int32_t depth;                       // steps taken so far
+    int64_t D;                           // elements per node
+    int32_t nchunks;                     // work items per node row
+    bool independent;                    // s = inf: xi_b = eta_b
+    float mix_shared, mix_innov;         // xi_b = mix_shared*xi_0 + mix_innov*eta_b
+    const float* mu;                     // bound linear velocity (device), or nullptr
+    float s0;
+    // scratch carving (device pointers inside buf.scratch)
+    int32_t* status;
+    unsigned int* counters;              // one ticket counter per (tree, node row)
+    double* partials;                    // [n_trees*nodes_cap][nchunks][3]
+};
+
+namespace bgrpo {
+
+// ---- streaming kernels (tree_step.cu) -------------------------------------------------------------------------
+struct StepLaunch {
+    float* latents;
+    const float* v;            // [n_trees][W_in][D] or nullptr
+    const float* mu;           // [n_trees][D] or nullptr
+    float* logp;
+    int32_t* table;            // SoA, stride = n_trees*nodes_cap
+    double* partials;
+    unsigned int* counters;
+    int64_t D;                 // elements per row
+    int32_t n_trees, nodes_cap, nchunks;
+    int32_t W_in, off_in, off_out, fan, step, is_split;
+    uint32_t node_id_base;     // tree_id_base * nodes_cap
+    uint32_t key0, key1;
+    float ca, cb;              // mean = ca*z + cb*x, x = v or mu
+    float g, inv_2g2, logp_const;
+    float mix_shared, mix_innov;
+    int32_t shared_noise;      // 1: finite s at a split step
+    int32_t write_children;    // 1: tree_step; 0: tree_logprob (children are read, nothing but logp is written)
+    float* logp_out;           // destination of the log-probs (== logp for tree_step)
+};
+cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s);
+cudaError_t launch_step(const StepLaunch& p, cudaStream_t s);
+
+struct RewardLaunch {
+    const float* latents; const float* target; float* r; double* partials; unsigned int* counters;
+    int64_t D; int32_t n_trees, nodes_cap, nchunks, leaves, off_leaf; float scale; int32_t mode;  // 0 mse, 1 cos
+};
+cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s);
+
+cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s);
+cudaError_t launch_philox_normals(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, float* out, int64_t n, cudaStream_t s);
+
+// ---- tree reductions (tree_reduce.cu) -------------------------------------------------------------------------
+struct FuseLaunch {
+    const float* leaf_r; const float* logp; float* rbar; float* adv; int32_t* status;
+    LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes; double beta_scaled; float eps, clip;
+};
+cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s);
+
+struct PruneLaunch {
+    const float* rbar; const int32_t* table; uint8_t* mask;
+    LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes, mode, k, last_split, ignore_last; uint64_t pruned_bits;
+};
+cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s);
+
+// ---- MLP velocity (mlp_velocity.cu) -----------------------------------------------------------------------------
+size_t mlp_packed_bytes(int hidden);
+cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, void* packed, cudaStream_t s);
+cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
+                       const void* packed, int hidden, float* v_out, cudaStream_t s);
+
+}  // namespace bgrpo

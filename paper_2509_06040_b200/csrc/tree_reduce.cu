@@ -1,0 +1,179 @@
+// Tree reductions: reward fusion (Eq. 3) + depth-wise normalisation (Eq. 4) in one kernel, and the width / depth
+// pruning masks ("Pruning Strategies") in another.  A tree has at most a few thousand nodes, so one CTA owns one
+// tree, keeps the per-node state in shared memory as doubles and walks the levels; the kernels are latency-bound.
+//
+// Fusion uses the bottom-up form of Eq. 3.  With a_c = beta*logp(c) the softmax weight of leaf l under node n
+// factorises along the path, so  S_n = sum_c e^{a_c} S_c,  R_n = sum_c e^{a_c} R_c,  rbar(n) = R_n / S_n  with
+// S_leaf = 1, R_leaf = r.  S is carried as log S (shifted by the largest term) so huge |beta*logp| cannot overflow;
+// R/S is carried directly as rbar:  rbar(n) = sum_c w_c rbar(c),  w_c = e^{a_c + logS_c - m} / sum_c' e^{a_c' + logS_c' - m}.
+#include "internal.h"
+
+namespace bgrpo {
+namespace {
+
+constexpr int kTreeThreads = 256;
+
+__device__ __forceinline__ double warp_sum_d(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__global__ void __launch_bounds__(kTreeThreads)
+fuse_advantage_kernel(const FuseLaunch p) {
+    extern __shared__ double sm[];
+    double* rb = sm;                 // rbar per node
+    double* ls = sm + p.nodes;       // log S per node
+    const int tree = blockIdx.x;
+    const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    const int T = p.T;
+    const int leaves = p.lv.width[T];
+    const int off_leaf = p.lv.offset[T];
+    __shared__ int bad;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    for (int l = threadIdx.x; l < leaves; l += kTreeThreads) {
+        const float r = p.leaf_r[static_cast<int64_t>(tree) * leaves + l];
+        if (!isfinite(r)) bad = 1;
+        rb[off_leaf + l] = static_cast<double>(r);
+        ls[off_leaf + l] = 0.0;
+    }
+    __syncthreads();
+    if (bad && threadIdx.x == 0) atomicOr(p.status, 1);
+    const double beta = p.beta_scaled;
+    for (int d = T - 1; d >= 0; --d) {
+        const int fan = p.lv.fanout[d];
+        const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
+        for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads) {
+            const int c0 = offc + j * fan;
+            double a[BGRPO_MAX_K];
+            double m = -INFINITY;
+#pragma unroll
+            for (int b = 0; b < BGRPO_MAX_K; ++b) {
+                if (b < fan) {
+                    a[b] = beta * static_cast<double>(p.logp[row0 + c0 + b]) + ls[c0 + b];
+                    m = fmax(m, a[b]);
+                }
+            }
+            double S = 0.0, R = 0.0;
+#pragma unroll
+            for (int b = 0; b < BGRPO_MAX_K; ++b) {
+                if (b < fan) {
+                    const double w = exp(a[b] - m);
+                    S += w;
+                    R += w * rb[c0 + b];
+                }
+            }
+            rb[off + j] = R / S;
+            ls[off + j] = m + log(S);
+        }
+        __syncthreads();
+    }
+    // Depth-wise statistics: one warp per depth, two passes (mean, then centred squares), fixed lane order.
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int d = warp; d <= T; d += kTreeThreads / 32) {
+        const int W = p.lv.width[d], off = p.lv.offset[d];
+        double s = 0.0;
+        for (int j = lane; j < W; j += 32) s += rb[off + j];
+        const double mean = warp_sum_d(s) / W;
+        double q = 0.0;
+        for (int j = lane; j < W; j += 32) { const double c = rb[off + j] - mean; q += c * c; }
+        const double sd = sqrt(warp_sum_d(q) / W);
+        const double inv = 1.0 / (sd + static_cast<double>(p.eps));
+        for (int j = lane; j < W; j += 32) {
+            double A = (d == 0) ? 0.0 : (rb[off + j] - mean) * inv;
+            if (p.clip > 0.0f) A = fmin(fmax(A, -static_cast<double>(p.clip)), static_cast<double>(p.clip));
+            p.adv[row0 + off + j] = static_cast<float>(A);
+            p.rbar[row0 + off + j] = static_cast<float>(rb[off + j]);
+        }
+    }
+}
+
+// rank of x among its siblings / leaves: number of entries that beat it (larger value, or equal value and lower index)
+__device__ __forceinline__ bool beats(float v_other, int i_other, float v_me, int i_me) {
+    return (v_other > v_me) || (v_other == v_me && i_other < i_me);
+}
+
+__global__ void __launch_bounds__(kTreeThreads)
+prune_kernel(const PruneLaunch p) {
+    extern __shared__ unsigned char keep[];            // per node
+    const int tree = blockIdx.x;
+    const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    const int T = p.T;
+    const float* rbar = p.rbar + row0;
+    if (p.mode == BGRPO_WIDTH_EXTREME_B) {
+        for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) keep[n] = 0;
+        __syncthreads();
+        const int L = p.lv.width[T], off = p.lv.offset[T];
+        const int64_t rows = static_cast<int64_t>(p.n_trees) * p.nodes_cap;
+        for (int l = threadIdx.x; l < L; l += kTreeThreads) {
+            const float v = rbar[off + l];
+            int better = 0, worse = 0;
+            for (int q = 0; q < L; ++q) {
+                const float u = rbar[off + q];
+                better += beats(u, q, v, l) ? 1 : 0;                       // rank from the top
+                worse += ((u < v) || (u == v && q < l)) ? 1 : 0;           // rank from the bottom
+            }
+            if (better < p.k || worse < p.k) {
+                int n = off + l;
+                for (int guard = 0; n >= 0 && guard <= T; ++guard) {       // root path through the node table
+                    keep[n] = 1;
+                    n = p.table[row0 + n];
+                }
+            }
+        }
+        (void)rows;
+        __syncthreads();
+    } else {
+        if (threadIdx.x == 0) keep[0] = 1;
+        __syncthreads();
+        for (int d = 0; d < T; ++d) {
+            const int fan = p.lv.fanout[d];
+            const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
+            const bool ranked = fan > 1 && (p.mode == BGRPO_WIDTH_PER_SPLIT_TOPK ||
+                                            (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && d == p.last_split));
+            for (int c = threadIdx.x; c < p.lv.width[d + 1]; c += kTreeThreads) {
+                const int j = c / fan, b = c - j * fan;
+                unsigned char k = keep[off + j];
+                if (ranked) {
+                    const float v = rbar[offc + c];
+                    int rank = 0;
+                    for (int q = 0; q < fan; ++q) rank += beats(rbar[offc + j * fan + q], q, v, b) ? 1 : 0;
+                    k = (k && rank < p.k) ? 1 : 0;
+                }
+                keep[offc + c] = k;
+            }
+            __syncthreads();
+        }
+    }
+    for (int d = 0; d <= T; ++d) {
+        const bool depth_ok = d > 0 && !((p.pruned_bits >> (d - 1)) & 1ull) && !(p.ignore_last && d == T);
+        const int off = p.lv.offset[d];
+        for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads)
+            p.mask[row0 + off + j] = (depth_ok && keep[off + j]) ? 1 : 0;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
+    const size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(fuse_advantage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    fuse_advantage_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s) {
+    const size_t smem = (static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    prune_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace bgrpo

@@ -1,0 +1,322 @@
+// Streaming kernels of the rollout: root initialisation, the fused gather / fork / Euler-Maruyama update /
+// log-prob step (Eq. 2 and the appendix's Euler-Maruyama form), the log-prob recompute under a given velocity,
+// and the leaf-reward reductions.  All of them are HBM-bound: every latent element is read or written once,
+// with 128-bit accesses, and the noise is generated in registers.
+//
+// Work decomposition: one CTA per (tree, parent node, chunk of kChunkVec float4).  A thread owns up to four
+// float4 of the parent row, loads them (and the velocity or target-mean operand) up front, evaluates the mean
+// once, and loops over the K children of the parent: the parent is read once however many children it has.
+// Sums over a row (log-prob, rewards) are float32 inside a thread's 16 elements, double from there on: warp
+// shuffles, shared memory across warps, one double per (row, chunk) in scratch, and the CTA that takes the last
+// ticket of a row adds the chunk partials in chunk order, so results do not depend on scheduling.
+#include "internal.h"
+#include "philox.cuh"
+
+namespace bgrpo {
+namespace {
+
+constexpr int kVecPerThread = kChunkVec / kStreamThreads;   // 4
+constexpr int kWarps = kStreamThreads / 32;
+constexpr int kPartialStride = 3;                           // doubles per (row, chunk) slot
+
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Publishes NV per-thread float sums of this CTA as doubles in partials[(row_b*nchunks + chunk)*3 + comp] and
+// returns true (to every thread) in the CTA that arrived last at `counter`.  rows: row_b = row0 + (v / comps).
+template <int NV>
+__device__ __forceinline__ bool publish_partials(const float (&acc)[NV], double* partials, unsigned int* counter,
+                                                 int64_t row0, int comps, int nchunks, int chunk) {
+    __shared__ double red[NV][kWarps];
+    __shared__ int last_flag;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const double s = warp_sum(static_cast<double>(acc[v]));
+        if (lane == 0) red[v][warp] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < NV) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
+        const int v = threadIdx.x;
+        const int64_t row = row0 + v / comps;
+        __stcg(&partials[(row * nchunks + chunk) * kPartialStride + (v % comps)], s);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int ticket = atomicAdd(counter, 1u);
+        last_flag = (ticket == static_cast<unsigned int>(nchunks) - 1u);
+        if (last_flag) *counter = 0u;     // every CTA of the row has arrived: leave the counter ready for the next launch
+    }
+    __syncthreads();
+    if (last_flag) __threadfence();
+    return last_flag != 0;
+}
+
+// Sum of one component of a row's chunk partials, in chunk order within each lane and a fixed shuffle tree across lanes.
+__device__ __forceinline__ double row_total(const double* partials, int64_t row, int comp, int nchunks) {
+    const int lane = threadIdx.x & 31;
+    double s = 0.0;
+    for (int c = lane; c < nchunks; c += 32) s += __ldcg(&partials[(row * nchunks + c) * kPartialStride + comp]);
+    s = warp_sum(s);
+    return __shfl_sync(0xffffffffu, s, 0);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Root: z_0 ~ N(0, I) from the ROOT stream, node-table row of the root, and a clean scratch (counters, status).
+__global__ void __launch_bounds__(kStreamThreads)
+root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters, int32_t* status, int64_t D,
+            int32_t n_trees, int32_t nodes_cap, int32_t nchunks, uint32_t node_id_base, uint32_t key0, uint32_t key1) {
+    const int chunk = blockIdx.x % nchunks;
+    const int tree = blockIdx.x / nchunks;
+    const int64_t D4 = D >> 2;
+    float4* z = reinterpret_cast<float4*>(latents + static_cast<int64_t>(tree) * nodes_cap * D);
+    const uint32_t gid = node_id_base + static_cast<uint32_t>(tree) * nodes_cap;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int64_t e = static_cast<int64_t>(chunk) * kChunkVec + k * kStreamThreads + threadIdx.x;
+        if (e < D4) z[e] = noise4(static_cast<uint32_t>(e), gid, 0u, BGRPO_TAG_ROOT, key0, key1);
+    }
+    const int64_t rows = static_cast<int64_t>(n_trees) * nodes_cap;
+    if (chunk == 0) {
+        for (int n = threadIdx.x; n < nodes_cap; n += kStreamThreads) counters[static_cast<int64_t>(tree) * nodes_cap + n] = 0u;
+        if (threadIdx.x == 0) {
+            const int64_t r = static_cast<int64_t>(tree) * nodes_cap;
+            table[r] = -1;
+            table[rows + r] = 0;
+            table[2 * rows + r] = -1;
+            table[3 * rows + r] = 0;
+            logp[r] = 0.0f;
+            if (tree == 0) *status = 0;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Fused step.  FAN children per parent; SHARED: xi_b mixes a per-parent xi_0 (finite s at a split step);
+// WRITE: true = tree_step (draw noise, write children), false = tree_logprob (read children, score them).
+template <int FAN, bool SHARED, bool WRITE>
+__global__ void __launch_bounds__(kStreamThreads)
+step_kernel(const StepLaunch p) {
+    const int chunk = blockIdx.x % p.nchunks;
+    const int row = blockIdx.x / p.nchunks;             // tree * W_in + j
+    const int tree = row / p.W_in;
+    const int j = row - tree * p.W_in;
+    const int64_t D4 = p.D >> 2;
+    const int64_t tree_row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    const int parent = p.off_in + j;
+    const int child0 = p.off_out + j * FAN;
+    const float4* __restrict__ zp = reinterpret_cast<const float4*>(p.latents + (tree_row0 + parent) * p.D);
+    const float4* __restrict__ xop = p.v ? reinterpret_cast<const float4*>(p.v + static_cast<int64_t>(row) * p.D)
+                                         : reinterpret_cast<const float4*>(p.mu + static_cast<int64_t>(tree) * p.D);
+    float4* zc = reinterpret_cast<float4*>(p.latents + (tree_row0 + child0) * p.D);
+    const uint32_t gid_parent = p.node_id_base + static_cast<uint32_t>(tree_row0 + parent);
+    const uint32_t gid_child0 = p.node_id_base + static_cast<uint32_t>(tree_row0 + child0);
+    const bool streamed_operand = (p.v != nullptr);
+
+    float acc[FAN];
+#pragma unroll
+    for (int b = 0; b < FAN; ++b) acc[b] = 0.0f;
+
+    const int64_t e0 = static_cast<int64_t>(chunk) * kChunkVec + threadIdx.x;
+    float4 z[kVecPerThread], x[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int64_t e = e0 + k * kStreamThreads;
+        if (e < D4) {
+            z[k] = __ldcs(zp + e);                                   // read once: evict first
+            x[k] = streamed_operand ? __ldcs(xop + e) : __ldg(xop + e);   // the target mean is shared by the whole level
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int64_t e = e0 + k * kStreamThreads;
+        if (e < D4) {
+            float4 m;
+            m.x = fmaf(p.ca, z[k].x, p.cb * x[k].x);
+            m.y = fmaf(p.ca, z[k].y, p.cb * x[k].y);
+            m.z = fmaf(p.ca, z[k].z, p.cb * x[k].z);
+            m.w = fmaf(p.ca, z[k].w, p.cb * x[k].w);
+            float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (WRITE && SHARED) xi0 = noise4(static_cast<uint32_t>(e), gid_parent, p.step, BGRPO_TAG_SHARED, p.key0, p.key1);
+#pragma unroll
+            for (int b = 0; b < FAN; ++b) {
+                float4 c;
+                if (WRITE) {
+                    float4 xi = noise4(static_cast<uint32_t>(e), gid_child0 + b, p.step, BGRPO_TAG_INNOV, p.key0, p.key1);
+                    if (SHARED) {
+                        xi.x = fmaf(p.mix_innov, xi.x, p.mix_shared * xi0.x);
+                        xi.y = fmaf(p.mix_innov, xi.y, p.mix_shared * xi0.y);
+                        xi.z = fmaf(p.mix_innov, xi.z, p.mix_shared * xi0.z);
+                        xi.w = fmaf(p.mix_innov, xi.w, p.mix_shared * xi0.w);
+                    }
+                    c.x = fmaf(p.g, xi.x, m.x);
+                    c.y = fmaf(p.g, xi.y, m.y);
+                    c.z = fmaf(p.g, xi.z, m.z);
+                    c.w = fmaf(p.g, xi.w, m.w);
+                    zc[static_cast<int64_t>(b) * D4 + e] = c;
+                } else {
+                    c = __ldcs(zc + static_cast<int64_t>(b) * D4 + e);
+                }
+                const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
+                acc[b] = fmaf(dx, dx, acc[b]);
+                acc[b] = fmaf(dy, dy, acc[b]);
+                acc[b] = fmaf(dz, dz, acc[b]);
+                acc[b] = fmaf(dw, dw, acc[b]);
+            }
+        }
+    }
+
+    const bool last = publish_partials<FAN>(acc, p.partials, &p.counters[tree_row0 + parent], tree_row0 + child0, 1,
+                                            p.nchunks, chunk);
+    if (!last) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp < FAN) {
+        const int b = warp;
+        const double ss = row_total(p.partials, tree_row0 + child0 + b, 0, p.nchunks);
+        if (lane == 0) {
+            const int64_t r = tree_row0 + child0 + b;
+            const double mean_sq = ss / static_cast<double>(p.D);
+            p.logp_out[r] = (p.g == 0.0f) ? 0.0f
+                                          : static_cast<float>(-mean_sq * static_cast<double>(p.inv_2g2) + static_cast<double>(p.logp_const));
+            if (WRITE) {
+                const int64_t rows = static_cast<int64_t>(p.n_trees) * p.nodes_cap;
+                const int64_t rp = tree_row0 + parent;
+                p.table[r] = parent;
+                p.table[rows + r] = p.step + 1;
+                p.table[2 * rows + r] = p.is_split ? p.step : p.table[2 * rows + rp];
+                p.table[3 * rows + r] = p.is_split ? b : p.table[3 * rows + rp];
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Leaf rewards: mode 0  r = -mean (z - target)^2 ; mode 1  r += scale * cos(z, target).
+template <int MODE>
+__global__ void __launch_bounds__(kStreamThreads)
+reward_kernel(const RewardLaunch p) {
+    const int chunk = blockIdx.x % p.nchunks;
+    const int row = blockIdx.x / p.nchunks;             // tree * leaves + l
+    const int tree = row / p.leaves;
+    const int l = row - tree * p.leaves;
+    const int64_t D4 = p.D >> 2;
+    const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + l;
+    const float4* __restrict__ z = reinterpret_cast<const float4*>(p.latents + node_row * p.D);
+    const float4* __restrict__ tg = reinterpret_cast<const float4*>(p.target + static_cast<int64_t>(tree) * p.D);
+    constexpr int NV = (MODE == 0) ? 1 : 3;
+    float acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = 0.0f;
+    const int64_t e0 = static_cast<int64_t>(chunk) * kChunkVec + threadIdx.x;
+    float4 a[kVecPerThread], t[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int64_t e = e0 + k * kStreamThreads;
+        if (e < D4) { a[k] = __ldcs(z + e); t[k] = __ldg(tg + e); }
+    }
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int64_t e = e0 + k * kStreamThreads;
+        if (e < D4) {
+            const float av[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
+            const float tv[4] = {t[k].x, t[k].y, t[k].z, t[k].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (MODE == 0) {
+                    const float d = av[q] - tv[q];
+                    acc[0] = fmaf(d, d, acc[0]);
+                } else {
+                    acc[0] = fmaf(av[q], tv[q], acc[0]);
+                    acc[1] = fmaf(av[q], av[q], acc[1]);
+                    acc[2] = fmaf(tv[q], tv[q], acc[2]);
+                }
+            }
+        }
+    }
+    const bool last = publish_partials<NV>(acc, p.partials, &p.counters[node_row], node_row, NV, p.nchunks, chunk);
+    if (!last) return;
+    if ((threadIdx.x >> 5) == 0) {
+        if (MODE == 0) {
+            const double ss = row_total(p.partials, node_row, 0, p.nchunks);
+            if (threadIdx.x == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
+        } else {
+            const double dot = row_total(p.partials, node_row, 0, p.nchunks);
+            const double zz = row_total(p.partials, node_row, 1, p.nchunks);
+            const double tt = row_total(p.partials, node_row, 2, p.nchunks);
+            if (threadIdx.x == 0)
+                p.r[row] = static_cast<float>(static_cast<double>(p.r[row]) + static_cast<double>(p.scale) * dot / (sqrt(zz) * sqrt(tt)));
+        }
+    }
+}
+
+__global__ void philox_words_kernel(uint32_t k0, uint32_t k1, uint32_t node, uint32_t step, uint32_t tag, uint4* out, int64_t nblk) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < nblk) out[i] = philox4x32_10(make_uint4(static_cast<uint32_t>(i), node, step, tag), k0, k1);
+}
+__global__ void philox_normals_kernel(uint32_t k0, uint32_t k1, uint32_t node, uint32_t step, uint32_t tag, float4* out, int64_t nblk) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < nblk) out[i] = noise4(static_cast<uint32_t>(i), node, step, tag, k0, k1);
+}
+
+template <int FAN>
+cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t s) {
+    if (!p.write_children) step_kernel<FAN, false, false><<<grid, kStreamThreads, 0, s>>>(p);
+    else if (p.shared_noise) step_kernel<FAN, true, true><<<grid, kStreamThreads, 0, s>>>(p);
+    else step_kernel<FAN, false, true><<<grid, kStreamThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s) {
+    const unsigned int grid = static_cast<unsigned int>(t->desc.n_trees) * t->nchunks;
+    root_kernel<<<grid, kStreamThreads, 0, s>>>(t->buf.latents, t->buf.node_table, t->buf.logp, t->counters, t->status, t->D,
+                                                t->desc.n_trees, t->desc.nodes_cap, t->nchunks,
+                                                static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap),
+                                                static_cast<uint32_t>(t->desc.seed), static_cast<uint32_t>(t->desc.seed >> 32));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_step(const StepLaunch& p, cudaStream_t s) {
+    const int64_t items = static_cast<int64_t>(p.n_trees) * p.W_in * p.nchunks;
+    if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    const unsigned int grid = static_cast<unsigned int>(items);
+    switch (p.fan) {
+        case 1: return launch_step_fan<1>(p, grid, s);
+        case 2: return launch_step_fan<2>(p, grid, s);
+        case 3: return launch_step_fan<3>(p, grid, s);
+        case 4: return launch_step_fan<4>(p, grid, s);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
+    const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * p.nchunks;
+    if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (p.mode == 0) reward_kernel<0><<<static_cast<unsigned int>(items), kStreamThreads, 0, s>>>(p);
+    else reward_kernel<1><<<static_cast<unsigned int>(items), kStreamThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {
+    if (nblk <= 0) return cudaSuccess;
+    philox_words_kernel<<<static_cast<unsigned int>((nblk + 255) / 256), 256, 0, s>>>(
+        static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), node, step, tag, reinterpret_cast<uint4*>(out), nblk);
+    return cudaGetLastError();
+}
+cudaError_t launch_philox_normals(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, float* out, int64_t n, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const int64_t nblk = n / 4;
+    philox_normals_kernel<<<static_cast<unsigned int>((nblk + 255) / 256), 256, 0, s>>>(
+        static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), node, step, tag, reinterpret_cast<float4*>(out), nblk);
+    return cudaGetLastError();
+}
+
+}  // namespace bgrpo

@@ -1,0 +1,58 @@
+"""Full-size parity in the launch configuration the benchmark times: the video-shaped tree
+(21x60x104 tokens x 16 channels, 111 nodes, closed-form velocity) is small enough for the
+oracle to compute whole, so every latent element, every log-prob, every reward, advantage and
+mask of the full workload is compared."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import credit, rewards
+from oracle import tree as otree
+from workloads import CONFIGS, make_inputs
+
+from test_gpu_parity import LATENT_TOL, LOGP_TOL, B, adv_close, assert_table, f32, oracle_rollout  # noqa: F401
+
+pytestmark = pytest.mark.gpu
+
+
+def test_video_config_whole_workload(B):
+    from paper_2509_06040_b200.session import TreeSession
+    w = CONFIGS["video"]
+    inp = make_inputs(w)
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+    s.run_all()
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    topo, lat, logp = oracle_rollout(w, inp, 1)
+    assert_table(s, topo, 1)
+    got = s.latents.cpu().numpy()
+    worst = 0.0
+    for n in range(topo.nodes):
+        worst = max(worst, float(np.abs(got[0, n] - lat[0, n]).max()))
+    assert worst <= LATENT_TOL, worst
+    assert np.abs(s.logp.cpu().numpy() - logp).max() <= LOGP_TOL
+    # siblings share their prefix: there is one stored row per node, and children of a split differ
+    for p in topo.level(5):
+        a, b = topo.children(p)
+        assert not np.array_equal(got[0, a], got[0, b])
+    r = np.array([rewards.neg_mse(lat[0][l], inp.target[0]) for l in topo.leaf_ids()])
+    got_r = s.leaf_r.cpu().numpy()[0]
+    assert np.abs(got_r - r).max() <= 1e-6 * np.abs(r).max()
+    # reductions, teacher-forced on the oracle's float32 rewards and log-probs
+    s.logp.copy_(torch.from_numpy(logp.astype(np.float32)))
+    s.leaf_r.copy_(torch.from_numpy(r.astype(np.float32)[None]))
+    s.fuse_advantage()
+    s.prune()
+    torch.cuda.synchronize()
+    r32 = r.astype(np.float32).astype(np.float64)
+    rbar = credit.fuse_rewards(topo, r32, logp[0].astype(np.float32).astype(np.float64), w.beta)
+    adv = credit.depth_advantages(topo, rbar, f32(w.eps))
+    assert adv_close(s.adv.cpu().numpy()[0], adv)
+    rbar32 = s.rbar.cpu().numpy()[0]
+    assert np.array_equal(rbar32, rbar.astype(np.float32))
+    mask = credit.gradient_mask(topo, rbar32, w.width_mode, w.width_k, (), w.ignore_last_step)
+    assert np.array_equal(s.mask.cpu().numpy()[0], mask)
+    assert int(mask.sum()) == sum(1 for n in range(1, topo.nodes) if mask[n])
+    # top-1 per split keeps exactly one leaf
+    assert int(mask[list(topo.leaf_ids())].sum()) == 1

@@ -1,0 +1,414 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, on the same seeded inputs.
+
+Tolerances (stated by the target): Philox integers, node table and masks bit-exact; latents and
+log-probs max abs error <= 1e-5; advantages <= 1e-4 relative (|d| <= 1e-4 * max(1, |A|)).
+Reductions are tested teacher-forced as well: the oracle's float32 log-probs / rewards / fused
+values are written into the device buffers, so the decision inputs are identical on both sides.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import credit, philox, rewards, sde
+from oracle import tree as otree
+from workloads import CONFIGS, Workload, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+LATENT_TOL = 1e-5
+LOGP_TOL = 1e-5
+ADV_RTOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def B():
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2509_06040_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _session(w, **kw):
+    from paper_2509_06040_b200.session import TreeSession
+    return TreeSession(w, **kw)
+
+
+def f32(x):
+    return float(np.float32(x))
+
+
+def oracle_rollout(w, inp, n_trees, tree_id_base=0, nodes_cap=None, velocity=None):
+    """Oracle latents [n_trees][nodes][D], logp [n_trees][nodes] for the linear-velocity workloads
+    (or any per-tree velocity callback factory `velocity(t)`)."""
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    lats, logps = [], []
+    for t in range(n_trees):
+        if velocity is None:
+            mu = inp.mu[t].astype(np.float64)
+            vel = lambda z, i, p, mu=mu: sde.linear_velocity(z.astype(np.float64), float(grid[i]), mu, f32(w.s0))
+        else:
+            vel = velocity(t)
+        lat, lp = sde.rollout(topo, w.D, grid, f32(w.sigma), w.branch_corr_s, w.seed, vel,
+                              tree_id=tree_id_base + t, nodes_cap=nodes_cap or topo.nodes)
+        lats.append(lat)
+        logps.append(lp)
+    return topo, np.stack(lats), np.stack(logps)
+
+
+def assert_table(s, topo, n_trees):
+    tab = s.node_table.cpu().numpy().reshape(4, n_trees, s.nodes_cap)
+    for t in range(n_trees):
+        assert np.array_equal(tab[0, t, :topo.nodes], topo.parent)
+        assert np.array_equal(tab[1, t, :topo.nodes], topo.depth)
+        assert np.array_equal(tab[2, t, :topo.nodes], topo.split_step)
+        assert np.array_equal(tab[3, t, :topo.nodes], topo.branch_id)
+
+
+def adv_close(got, ref):
+    return np.all(np.abs(got - ref) <= ADV_RTOL * np.maximum(1.0, np.abs(ref)))
+
+
+# ---------------------------------------------------------------------------------------------- noise
+def test_philox_integer_stream_bit_exact(B):
+    for seed, node, step, tag, nblk in ((0, 0, 0, 0, 64), (1223627, 154, 15, 2, 32400), ((7 << 32) | 9, 2 ** 32 - 1, 19, 1, 1000)):
+        out = torch.empty((nblk, 4), dtype=torch.int32, device="cuda")
+        B.philox_words_fill(seed, node, step, tag, out, nblk)
+        got = out.cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, philox.noise_words(seed, node, step, tag, 4 * nblk))
+
+
+def test_normals_match_float64_transform(B):
+    n = 1 << 22
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    B.philox_normal_fill(42, 77, 3, 2, out, n)
+    got = out.cpu().numpy().astype(np.float64)
+    ref = philox.node_noise(42, 77, 3, 2, n)
+    err = np.abs(got - ref)
+    # g <= 0.3 in every workload, so 2e-5 on xi is < 1e-5 on a latent; the observed error is far smaller
+    assert err.max() < 2e-5, err.max()
+    # the rare words whose uniform sits next to 1 (tiny radius) and next to 0 (largest radius) are present and accurate
+    w = philox.noise_words(42, 77, 3, 2, n)
+    ua = philox.uniform_open(w[:, 0])
+    near_one = np.nonzero(1 - ua < 2.0 ** -9)[0]
+    assert len(near_one) > 100 and err.reshape(-1, 4)[near_one].max() < 2e-5
+    assert err.reshape(-1, 4)[np.argmin(ua)].max() < 2e-5
+
+
+# ---------------------------------------------------------------------------------------------- toy config, end to end
+def test_toy_config_end_to_end(B):
+    w = CONFIGS["toy"]
+    inp = make_inputs(w)
+    s = _session(w)
+    s.upload_inputs(inp)
+    s.run_all()
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    topo, lat, logp = oracle_rollout(w, inp, 1)
+    assert_table(s, topo, 1)
+    assert np.abs(s.latents.cpu().numpy() - lat).max() <= LATENT_TOL
+    assert np.abs(s.logp.cpu().numpy() - logp).max() <= LOGP_TOL
+    r = np.array([rewards.neg_mse(lat[0][l], inp.mu[0]) for l in topo.leaf_ids()])
+    assert np.abs(s.leaf_r.cpu().numpy()[0] - r).max() <= 1e-5
+    rbar = credit.fuse_rewards(topo, r, logp[0], w.beta)
+    adv = credit.depth_advantages(topo, rbar, f32(w.eps))
+    assert np.abs(s.rbar.cpu().numpy()[0] - rbar).max() <= 1e-5
+    assert adv_close(s.adv.cpu().numpy()[0], adv)
+    assert np.array_equal(s.mask.cpu().numpy()[0], credit.gradient_mask(topo, rbar, w.width_mode, w.width_k))
+    st = B.tree_stats(s.tree)
+    assert (st["nodes"], st["node_steps"], st["model_evals"], st["frontier_width"]) == (13, 12, 9, 4)
+    assert B.tree_levels(s.tree) == (topo.width, topo.offset[:-1])
+
+
+# ---------------------------------------------------------------------------------------------- tiles, tails, K, s, batches
+RAGGED = [
+    # name, n_trees, tokens, channels, T, K, splits, sigma, s, tree_id_base, extra cap
+    ("two_chunks_tail_k3_corr", 3, 2125, 4, 5, 3, (1, 3), 0.3, 2.0, 5, 7),
+    ("k4_independent", 2, 1031, 4, 4, 4, (0, 3), 0.5, math.inf, 0, 0),
+    ("k2_corr_s4_every_step", 1, 300, 4, 4, 2, (0, 1, 2, 3), 0.3, 4.0, 1000, 3),
+    ("no_split_k1", 2, 9, 4, 6, 1, (), 0.7, math.inf, 0, 0),
+    ("deterministic_sigma0", 1, 520, 4, 4, 2, (0, 2), 0.0, 1.0, 0, 0),
+    ("exact_chunk_multiple", 1, 2048, 4, 3, 2, (1,), 0.3, math.inf, 2, 0),
+]
+
+
+@pytest.mark.parametrize("case", RAGGED, ids=[c[0] for c in RAGGED])
+def test_rollout_parity_over_tiles_and_tails(B, case):
+    name, n_trees, tokens, channels, T, K, splits, sigma, s_corr, base, extra = case
+    w = Workload(name=name, n_trees=n_trees, tokens=tokens, channels=channels, T=T, K=K, splits=splits, sigma=sigma,
+                 velocity="linear", reward="neg_mse_mu", branch_corr_s=s_corr, seed=991 + T)
+    inp = make_inputs(w, tree_base=base)
+    cap = w.nodes + extra
+    s = _session(w, tree_id_base=base, nodes_cap=cap)
+    s.upload_inputs(inp)
+    s.latents.fill_(float("nan"))
+    s.run_all()
+    torch.cuda.synchronize()
+    topo, lat, logp = oracle_rollout(w, inp, n_trees, tree_id_base=base, nodes_cap=cap)
+    assert_table(s, topo, n_trees)
+    got = s.latents.cpu().numpy()[:, :topo.nodes]
+    assert np.abs(got - lat).max() <= LATENT_TOL
+    assert np.abs(s.logp.cpu().numpy()[:, :topo.nodes] - logp).max() <= LOGP_TOL
+    if extra:
+        assert np.all(np.isnan(s.latents.cpu().numpy()[:, topo.nodes:]))      # rows beyond the tree are never written
+    for t in range(n_trees):
+        r = np.array([rewards.neg_mse(lat[t][l], inp.mu[t]) for l in topo.leaf_ids()])
+        assert np.abs(s.leaf_r.cpu().numpy()[t] - r).max() <= 1e-5 * max(1.0, np.abs(r).max())
+    # running the same handle again with the same seed reproduces every bit (fixed reduction order)
+    first_lat, first_logp = s.latents.clone(), s.logp.clone()
+    s.rollout()
+    torch.cuda.synchronize()
+    assert torch.equal(first_logp[:, :topo.nodes], s.logp[:, :topo.nodes])
+    assert torch.equal(first_lat[:, :topo.nodes], s.latents[:, :topo.nodes])
+    # and another seed gives another tree
+    s.rollout(seed=12345)
+    torch.cuda.synchronize()
+    if sigma > 0:
+        assert not torch.equal(first_lat[:, :topo.nodes], s.latents[:, :topo.nodes])
+
+
+def test_sharded_batch_draws_the_same_noise(B):
+    """Trees are independent: a shard with tree_id_base = t reproduces tree t of the whole batch."""
+    w = Workload(name="shard", n_trees=4, tokens=64, channels=4, T=3, K=2, splits=(0, 2), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    whole = _session(w)
+    whole.upload_inputs(make_inputs(w))
+    whole.rollout()
+    part = _session(w.scaled(n_trees=2), tree_id_base=2)
+    part.upload_inputs(make_inputs(w.scaled(n_trees=2), tree_base=2))
+    part.rollout()
+    torch.cuda.synchronize()
+    assert torch.equal(whole.latents[2:], part.latents)
+    assert torch.equal(whole.logp[2:], part.logp)
+
+
+# ---------------------------------------------------------------------------------------------- given velocity (MLP stand-in path)
+def test_step_with_supplied_velocity_and_logprob_recompute(B):
+    """tree_step with a velocity buffer (the MLP configurations' path), teacher-forced: the oracle's MLP
+    produces v for every frontier, both sides consume the same float32 v."""
+    from oracle import mlp
+    w = Workload(name="given_v", n_trees=2, tokens=40, channels=64, T=3, K=2, splits=(0, 2), sigma=0.3,
+                 velocity="mlp", reward="mixture", hidden=128)
+    inp = make_inputs(w)
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    v_store = {}
+
+    def vel_factory(t):
+        def vel(z, i, p):
+            v = mlp.mlp_velocity(z.reshape(w.tokens, w.channels), inp.W1, inp.W2).reshape(-1)
+            v_store[(t, i, p)] = v
+            return v
+        return vel
+
+    lat, logp = [], []
+    for t in range(w.n_trees):
+        a, b = sde.rollout(topo, w.D, grid, f32(w.sigma), w.branch_corr_s, w.seed, vel_factory(t), tree_id=t, nodes_cap=topo.nodes)
+        lat.append(a)
+        logp.append(b)
+    lat, logp = np.stack(lat), np.stack(logp)
+
+    from paper_2509_06040_b200.session import TreeSession
+    s = TreeSession(w)
+    s.init()
+    v_bufs = []
+    for i in range(w.T):
+        v = np.stack([np.stack([v_store[(t, i, p)] for p in topo.level(i)]) for t in range(w.n_trees)])
+        v_dev = torch.from_numpy(v).cuda()
+        v_bufs.append(v_dev)
+        B.tree_step(s.tree, 1 if i in w.splits else 0, v_dev)
+    torch.cuda.synchronize()
+    assert np.abs(s.latents.cpu().numpy() - lat).max() <= LATENT_TOL
+    assert np.abs(s.logp.cpu().numpy() - logp).max() <= LOGP_TOL
+    # recompute under the same velocity: rho = 1
+    out = torch.zeros_like(s.logp)
+    for i in range(w.T):
+        B.tree_logprob(s.tree, i, v_bufs[i], out)
+    torch.cuda.synchronize()
+    assert (out - s.logp).abs()[:, 1:].max().item() <= LOGP_TOL
+    # under another velocity (a perturbed one): matches the oracle's edge log-prob of the stored latents
+    i = 1
+    v_new = v_bufs[i] + 0.05
+    out2 = torch.full_like(s.logp, 7.0)
+    B.tree_logprob(s.tree, i, v_new, out2)
+    torch.cuda.synchronize()
+    got = out2.cpu().numpy()
+    v_new_h = v_new.cpu().numpy()
+    for t in range(w.n_trees):
+        for j, p in enumerate(topo.level(i)):
+            for c in topo.children(p):
+                ref = sde.edge_logp(lat[t][p], lat[t][c], v_new_h[t, j], grid[i], grid[i] - grid[i + 1], f32(w.sigma))
+                assert abs(got[t, c] - ref) <= LOGP_TOL
+        untouched = [n for n in range(topo.nodes) if topo.depth[n] != i + 1]
+        assert np.all(got[t, untouched] == 7.0)
+
+
+def test_logprob_all_edges_linear_velocity(B):
+    w = Workload(name="lp_all", n_trees=2, tokens=700, channels=4, T=4, K=2, splits=(0, 2), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    inp = make_inputs(w)
+    s = _session(w)
+    s.upload_inputs(inp)
+    s.rollout()
+    out = torch.zeros_like(s.logp)
+    B.tree_logprob(s.tree, -1, None, out)
+    torch.cuda.synchronize()
+    assert (out - s.logp)[:, 1:].abs().max().item() <= LOGP_TOL
+    topo, lat, logp = oracle_rollout(w, inp, 2)
+    assert np.abs(out.cpu().numpy()[:, 1:] - logp[:, 1:]).max() <= LOGP_TOL
+    # a different policy (another target mean) against the oracle
+    mu2 = torch.from_numpy(inp.mu + 0.1).cuda()
+    B.velocity_linear_bind(s.tree, mu2, 0.5)
+    B.tree_logprob(s.tree, -1, None, out)
+    torch.cuda.synchronize()
+    grid = w.t_grid().astype(np.float64)
+    got = out.cpu().numpy()
+    for t in range(2):
+        mu_h = (inp.mu[t] + np.float32(0.1)).astype(np.float64)
+        for c in range(1, topo.nodes):
+            p, i = int(topo.parent[c]), int(topo.depth[c]) - 1
+            v = sde.linear_velocity(lat[t][p].astype(np.float64), grid[i], mu_h, 0.5)
+            ref = sde.edge_logp(lat[t][p], lat[t][c], v, grid[i], grid[i] - grid[i + 1], f32(w.sigma))
+            assert abs(got[t, c] - ref) <= 2e-5 * max(1.0, abs(ref))
+
+
+# ---------------------------------------------------------------------------------------------- rewards
+def test_leaf_rewards(B):
+    w = Workload(name="rw", n_trees=3, tokens=1500, channels=4, T=2, K=3, splits=(0, 1), sigma=0.3,
+                 velocity="linear", reward="normal_plus_cos")
+    inp = make_inputs(w)
+    s = _session(w)
+    s.upload_inputs(inp)
+    s.rollout()
+    s.rewards()
+    torch.cuda.synchronize()
+    topo, lat, _ = oracle_rollout(w, inp, 3)
+    got = s.leaf_r.cpu().numpy()
+    for t in range(3):
+        for q, l in enumerate(topo.leaf_ids()):
+            ref = float(inp.reward_draws[t, q]) + 0.1 * rewards.cosine(lat[t][l], inp.target[t])
+            assert abs(got[t, q] - ref) <= 1e-6 * max(1.0, abs(ref))
+    B.leaf_reward_mse(s.tree, s.target, s.leaf_r)
+    torch.cuda.synchronize()
+    got = s.leaf_r.cpu().numpy()
+    for t in range(3):
+        for q, l in enumerate(topo.leaf_ids()):
+            ref = rewards.neg_mse(lat[t][l], inp.target[t])
+            assert abs(got[t, q] - ref) <= 1e-6 * max(1.0, abs(ref))
+
+
+# ---------------------------------------------------------------------------------------------- reductions, teacher-forced
+def _grown_session(B, T, K, splits, n_trees=2, D_tokens=16):
+    w = Workload(name="red", n_trees=n_trees, tokens=D_tokens, channels=4, T=T, K=K, splits=splits, sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    s = _session(w)
+    s.upload_inputs(make_inputs(w))
+    s.rollout()
+    return w, s, otree.build_topology(T, K, splits)
+
+
+@pytest.mark.parametrize("T,K,splits", [(16, 2, (0, 3, 6, 9)), (6, 3, (0, 2, 5)), (5, 4, (1, 2, 4)), (20, 2, (0, 2, 4, 6, 8, 10)), (3, 2, ())])
+def test_fuse_and_advantage_against_enumeration(B, T, K, splits):
+    w, s, topo = _grown_session(B, T, K, splits)
+    rng = np.random.default_rng(T * 10 + K)
+    r = rng.standard_normal((2, topo.leaves)).astype(np.float32)
+    r[1] = 3.0 + 1e-3 * r[1]                       # a tree whose rewards differ in the 4th digit only
+    lp = (-np.abs(rng.standard_normal((2, topo.nodes))) - 0.3).astype(np.float32)
+    lp[:, 0] = 0
+    s.logp.copy_(torch.from_numpy(lp))
+    r_dev = torch.from_numpy(r).cuda()
+    for beta, scale, eps, clip in ((0.0, 1.0, 1e-6, 0.0), (1.0, 1.0, 1e-6, 0.0), (0.5, 64.0, 1e-3, 0.0), (1.0, 1.0, 1e-6, 0.8), (1.0, 1e5, 1e-6, 0.0)):
+        B.tree_fuse_advantage(s.tree, r_dev, beta, scale, eps, clip)
+        torch.cuda.synchronize()
+        for t in range(2):
+            rbar = credit.fuse_rewards(topo, r[t], lp[t].astype(np.float64), beta, scale)
+            adv = credit.depth_advantages(topo, rbar, f32(eps), clip)
+            got_rbar = s.rbar.cpu().numpy()[t]
+            assert np.abs(got_rbar - rbar).max() <= 1e-6 * max(1.0, np.abs(rbar).max())
+            assert adv_close(s.adv.cpu().numpy()[t], adv), (beta, scale, t)
+            assert s.adv.cpu().numpy()[t, 0] == 0.0
+    B.tree_sync_status(s.tree)
+
+
+@pytest.mark.parametrize("T,K,splits", [(16, 2, (0, 3, 6, 9)), (6, 4, (0, 2, 5)), (5, 3, (1, 2, 4)), (20, 2, (0, 5, 10))])
+def test_prune_masks_bit_exact(B, T, K, splits):
+    w, s, topo = _grown_session(B, T, K, splits)
+    rng = np.random.default_rng(T + K)
+    rbar = rng.standard_normal((2, topo.nodes)).astype(np.float32)
+    rbar[1] = np.round(rbar[1])                    # many exact ties
+    s.rbar.copy_(torch.from_numpy(rbar))
+    before_adv, before_lat = s.adv.clone(), s.latents.clone()
+    pruned = sorted(rng.choice(T, size=min(4, T), replace=False).tolist())
+    cases = [(B.WIDTH_NONE, 0, (), False), (B.WIDTH_PER_SPLIT_TOPK, 1, (), False), (B.WIDTH_PER_SPLIT_TOPK, 2, pruned, False),
+             (B.WIDTH_LAST_SPLIT_TOPK, 1, (), True), (B.WIDTH_EXTREME_B, 1, (), False), (B.WIDTH_EXTREME_B, 3, pruned, True),
+             (B.WIDTH_EXTREME_B, 10 ** 6, (), False), (B.WIDTH_PER_SPLIT_TOPK, K, pruned, False)]
+    for mode, k, pr, ign in cases:
+        s.mask.fill_(9)
+        B.tree_prune(s.tree, mode, k, pr, ign)
+        torch.cuda.synchronize()
+        got = s.mask.cpu().numpy()
+        for t in range(2):
+            ref = credit.gradient_mask(topo, rbar[t], mode, k, pr, ign)
+            assert np.array_equal(got[t], ref), (mode, k, pr, ign, t)
+    # pruning writes the mask only
+    assert torch.equal(s.rbar.cpu(), torch.from_numpy(rbar))
+    assert torch.equal(before_adv, s.adv) and torch.equal(before_lat, s.latents)
+
+
+# ---------------------------------------------------------------------------------------------- states and errors
+def test_state_and_capacity_errors(B):
+    w = Workload(name="err", n_trees=1, tokens=16, channels=4, T=3, K=2, splits=(0, 1, 2), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    inp = make_inputs(w)
+    s = _session(w, nodes_cap=11)                  # the full tree would need 15 rows
+    s.upload_inputs(inp)
+    s.init()
+    r = torch.zeros((1, 8), device="cuda")
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_fuse_advantage(s.tree, r)
+    assert e.value.status == B.ERR_STATE
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_prune(s.tree, B.WIDTH_NONE, 0)
+    assert e.value.status == B.ERR_STATE
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_logprob(s.tree, 0, None, s.logp)
+    assert e.value.status == B.ERR_STATE
+    B.tree_step(s.tree, 1)
+    B.tree_step(s.tree, 1)
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_step(s.tree, 1)                     # 1 + 2 + 4 + 8 > 11
+    assert e.value.status == B.ERR_CAPACITY
+    B.tree_step(s.tree, 0)                         # the refused call left the tree usable: 7 + 4 rows fit
+    torch.cuda.synchronize()
+    assert B.tree_stats(s.tree)["nodes"] == 11
+
+
+def test_step_past_depth_and_missing_velocity(B):
+    w = Workload(name="err2", n_trees=1, tokens=16, channels=4, T=2, K=2, splits=(0,), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    s = _session(w)
+    s.init()                                        # no velocity bound
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_step(s.tree, 1)
+    assert e.value.status == B.ERR_STATE
+    s.upload_inputs(make_inputs(w))
+    B.velocity_linear_bind(s.tree, s.mu, 0.5)
+    B.tree_step(s.tree, 1)
+    B.tree_step(s.tree, 0)
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_step(s.tree, 0)
+    assert e.value.status == B.ERR_STATE
+    torch.cuda.synchronize()
+
+
+def test_nonfinite_reward_sets_status(B):
+    w, s, topo = _grown_session(B, 3, 2, (0, 1), n_trees=1)
+    r = torch.tensor([[0.0, 1.0, float("nan"), 2.0]], device="cuda")
+    B.tree_fuse_advantage(s.tree, r)
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_sync_status(s.tree)
+    assert e.value.status == B.ERR_NONFINITE
+    B.tree_sync_status(s.tree)                     # the word is cleared by the read
