@@ -309,32 +309,36 @@ def run_ours(args, w):
         t_step = np.zeros(w.T)
         t_mlp = np.zeros(w.T)
         t_other = 0.0
-        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        def evs(n):
+            return [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+
         for rep in range(reps):
+            # events are recorded back to back on the launching stream and read after one final synchronize,
+            # so an interval holds one launch (plus its in-stream launch gap), never a host round trip
             if flush:
                 flush_buf.fill_(1.0)
-            a.record()
+            e_init, e_tail = evs(2), evs(2)
+            e_lvl = [evs(3) for _ in range(w.T)]
+            e_init[0].record()
             s.init(seed=w.seed + 3000 + rep)
-            b.record()
-            b.synchronize()
-            t_other += a.elapsed_time(b)
+            e_init[1].record()
             for i in range(w.T):
-                a.record()
+                e_lvl[i][0].record()
                 if w.velocity == "mlp":
                     B.velocity_mlp(s.tree, s.packed, w.hidden, s.v)
-                b.record()
+                e_lvl[i][1].record()
                 B.tree_step(s.tree, 1 if i in w.splits else 0, s.v if w.velocity == "mlp" else None)
-                c.record()
-                c.synchronize()
-                t_mlp[i] += a.elapsed_time(b)
-                t_step[i] += b.elapsed_time(c)
-            a.record()
+                e_lvl[i][2].record()
+            e_tail[0].record()
             s.rewards()
             s.fuse_advantage()
             s.prune()
-            b.record()
-            b.synchronize()
-            t_other += a.elapsed_time(b)
+            e_tail[1].record()
+            torch.cuda.synchronize()
+            t_other += e_init[0].elapsed_time(e_init[1]) + e_tail[0].elapsed_time(e_tail[1])
+            for i in range(w.T):
+                t_mlp[i] += e_lvl[i][0].elapsed_time(e_lvl[i][1]) if w.velocity == "mlp" else 0.0
+                t_step[i] += e_lvl[i][1].elapsed_time(e_lvl[i][2])
         t_step /= reps
         t_mlp /= reps
         t_other /= reps
@@ -398,8 +402,8 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="video", choices=list(CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")

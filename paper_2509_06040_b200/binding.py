@@ -118,7 +118,7 @@ class Tree:
     keep: tuple
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and lib is not None:     # `lib` is gone at interpreter shutdown
             lib.bgrpo_tree_destroy(self.handle)
             self.handle = None
 

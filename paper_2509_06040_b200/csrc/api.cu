@@ -225,8 +225,7 @@ static void fill_step_launch(const bgrpo_tree* t, int step, const float* v_dev, 
     p->nchunks = t->nchunks;
     p->step = step;
     p->node_id_base = static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap);
-    p->key0 = static_cast<uint32_t>(t->desc.seed);
-    p->key1 = static_cast<uint32_t>(t->desc.seed >> 32);
+    p->keys = make_philox_keys(t->desc.seed);
     p->ca = v_dev ? k.a : k.lin_a;
     p->cb = v_dev ? k.b : k.lin_b;
     p->g = k.g;

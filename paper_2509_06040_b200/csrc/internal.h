@@ -12,6 +12,29 @@ constexpr int kChunkVec = 1024;        // float4 per (parent, chunk) work item o
 constexpr int kStreamThreads = 256;    // threads per CTA of the streaming kernels
 constexpr int kScratchHeader = 256;    // bytes reserved at the start of scratch for the status word
 
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;   // Philox4x32 multipliers and Weyl key increments (Salmon et al., SC'11)
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+// The ten round keys of a 64-bit seed: key r = (k0 + r*W0, k1 + r*W1).  They are the same for every thread of
+// a launch, so the host computes them once and the kernels read them as launch constants.
+struct PhiloxKeys {
+    uint32_t k[10][2];
+};
+
+inline PhiloxKeys make_philox_keys(uint64_t seed) {
+    PhiloxKeys out;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        out.k[r][0] = k0;
+        out.k[r][1] = k1;
+        k0 += kPhiloxW0;
+        k1 += kPhiloxW1;
+    }
+    return out;
+}
+
 // Per-step scalars of the Euler-Maruyama mean and the Gaussian transition, computed in double on the host.
 //   mean = a*z + b*v                       (v given)
 //        = lin_a*z + lin_b*mu              (closed-form velocity v = k z - (1 + k(1-t)) mu folded in)
@@ -65,7 +88,7 @@ struct StepLaunch {
     int32_t n_trees, nodes_cap, nchunks;
     int32_t W_in, off_in, off_out, fan, step, is_split;
     uint32_t node_id_base;     // tree_id_base * nodes_cap
-    uint32_t key0, key1;
+    PhiloxKeys keys;
     float ca, cb;              // mean = ca*z + cb*x, x = v or mu
     float g, inv_2g2, logp_const;
     float mix_shared, mix_innov;

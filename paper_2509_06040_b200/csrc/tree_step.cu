@@ -6,9 +6,10 @@
 // Work decomposition: one CTA per (tree, parent node, chunk of kChunkVec float4).  A thread owns up to four
 // float4 of the parent row, loads them (and the velocity or target-mean operand) up front, evaluates the mean
 // once, and loops over the K children of the parent: the parent is read once however many children it has.
-// Sums over a row (log-prob, rewards) are float32 inside a thread's 16 elements, double from there on: warp
-// shuffles, shared memory across warps, one double per (row, chunk) in scratch, and the CTA that takes the last
-// ticket of a row adds the chunk partials in chunk order, so results do not depend on scheduling.
+// Sums over a row (log-prob, rewards) are float32 inside a thread's 16 elements (inside a warp's 512 for the
+// log-prob), double from there on: shared memory across warps, one double per (row, chunk) in scratch, and the
+// CTA that takes the last ticket of a row adds the chunk partials in a fixed order, so results do not depend
+// on scheduling.
 #include "internal.h"
 #include "philox.cuh"
 
@@ -25,41 +26,54 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-// Publishes NV per-thread float sums of this CTA as doubles in partials[(row_b*nchunks + chunk)*3 + comp] and
-// returns true (to every thread) in the CTA that arrived last at `counter`.  rows: row_b = row0 + (v / comps).
-template <int NV>
+// Publishes NV per-thread float sums of this CTA as doubles in partials[(row_b*nchunks + chunk)*3 + comp]
+// (row_b = row0 + v / comps) and takes a ticket on `counter`.  Only warp 0 returns with a meaningful value: true in
+// the CTA whose ticket was the row's last, after which every chunk partial of the row is visible to it.  The other
+// warps have nothing left to do once their sums are in shared memory.  Sums are float inside a warp (WARP_FLOAT:
+// 512 elements, a fixed shuffle tree) or double from the thread level on, and double across warps and chunks.
+template <int NV, bool WARP_FLOAT>
 __device__ __forceinline__ bool publish_partials(const float (&acc)[NV], double* partials, unsigned int* counter,
                                                  int64_t row0, int comps, int nchunks, int chunk) {
     __shared__ double red[NV][kWarps];
-    __shared__ int last_flag;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
-        const double s = warp_sum(static_cast<double>(acc[v]));
+        double s;
+        if (WARP_FLOAT) {
+            float f = acc[v];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) f += __shfl_down_sync(0xffffffffu, f, o);
+            s = static_cast<double>(f);
+        } else {
+            s = warp_sum(static_cast<double>(acc[v]));
+        }
         if (lane == 0) red[v][warp] = s;
     }
     __syncthreads();
-    if (threadIdx.x < NV) {
-        double s = 0.0;
+    if (warp != 0) return false;
+    int last = 0;
+    if (lane == 0) {
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
-        const int v = threadIdx.x;
-        const int64_t row = row0 + v / comps;
-        __stcg(&partials[(row * nchunks + chunk) * kPartialStride + (v % comps)], s);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
+        for (int v = 0; v < NV; ++v) {
+            double s = 0.0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) s += red[v][w];
+            const int64_t row = row0 + v / comps;
+            __stcg(&partials[(row * nchunks + chunk) * kPartialStride + (v % comps)], s);
+        }
+        __threadfence();
         const unsigned int ticket = atomicAdd(counter, 1u);
-        last_flag = (ticket == static_cast<unsigned int>(nchunks) - 1u);
-        if (last_flag) *counter = 0u;     // every CTA of the row has arrived: leave the counter ready for the next launch
+        last = (ticket == static_cast<unsigned int>(nchunks) - 1u);
+        if (last) {
+            *counter = 0u;        // every CTA of the row has arrived: leave the counter ready for the next launch
+            __threadfence();
+        }
     }
-    __syncthreads();
-    if (last_flag) __threadfence();
-    return last_flag != 0;
+    return __shfl_sync(0xffffffffu, last, 0) != 0;
 }
 
-// Sum of one component of a row's chunk partials, in chunk order within each lane and a fixed shuffle tree across lanes.
+// Sum of one component of a row's chunk partials, in chunk order within each lane and a fixed shuffle tree across
+// lanes.  Called by whole warps only.
 __device__ __forceinline__ double row_total(const double* partials, int64_t row, int comp, int nchunks) {
     const int lane = threadIdx.x & 31;
     double s = 0.0;
@@ -72,7 +86,7 @@ __device__ __forceinline__ double row_total(const double* partials, int64_t row,
 // Root: z_0 ~ N(0, I) from the ROOT stream, node-table row of the root, and a clean scratch (counters, status).
 __global__ void __launch_bounds__(kStreamThreads)
 root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters, int32_t* status, int64_t D,
-            int32_t n_trees, int32_t nodes_cap, int32_t nchunks, uint32_t node_id_base, uint32_t key0, uint32_t key1) {
+            int32_t n_trees, int32_t nodes_cap, int32_t nchunks, uint32_t node_id_base, const __grid_constant__ PhiloxKeys keys) {
     const int chunk = blockIdx.x % nchunks;
     const int tree = blockIdx.x / nchunks;
     const int64_t D4 = D >> 2;
@@ -81,7 +95,7 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int64_t e = static_cast<int64_t>(chunk) * kChunkVec + k * kStreamThreads + threadIdx.x;
-        if (e < D4) z[e] = noise4(static_cast<uint32_t>(e), gid, 0u, BGRPO_TAG_ROOT, key0, key1);
+        if (e < D4) z[e] = noise4(static_cast<uint32_t>(e), gid, 0u, BGRPO_TAG_ROOT, keys);
     }
     const int64_t rows = static_cast<int64_t>(n_trees) * nodes_cap;
     if (chunk == 0) {
@@ -100,15 +114,69 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
 
 // ---------------------------------------------------------------------------------------------------------------
 // Fused step.  FAN children per parent; SHARED: xi_b mixes a per-parent xi_0 (finite s at a split step);
-// WRITE: true = tree_step (draw noise, write children), false = tree_logprob (read children, score them).
+// WRITE: true = tree_step (draw noise, write children), false = tree_logprob (read children, score them);
+// FULL: the CTA's chunk lies wholly inside the row, so no element needs a bounds test.
+template <int FAN, bool SHARED, bool WRITE, bool FULL>
+__device__ __forceinline__ void step_elements(const StepLaunch& p, const float4* __restrict__ zp, const float4* __restrict__ xop,
+                                              float4* zc, uint32_t e0, uint32_t D4, uint32_t gid_parent, uint32_t gid_child0,
+                                              bool streamed_operand, float (&acc)[FAN]) {
+    float4 z[kVecPerThread], x[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const uint32_t e = e0 + k * kStreamThreads;
+        if (FULL || e < D4) {
+            z[k] = __ldcs(zp + e);                                        // read once: evict first
+            x[k] = streamed_operand ? __ldcs(xop + e) : __ldg(xop + e);   // the target mean is shared by the whole level
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const uint32_t e = e0 + k * kStreamThreads;
+        if (FULL || e < D4) {
+            float4 m;
+            m.x = fmaf(p.ca, z[k].x, p.cb * x[k].x);
+            m.y = fmaf(p.ca, z[k].y, p.cb * x[k].y);
+            m.z = fmaf(p.ca, z[k].z, p.cb * x[k].z);
+            m.w = fmaf(p.ca, z[k].w, p.cb * x[k].w);
+            float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (WRITE && SHARED) xi0 = noise4(e, gid_parent, p.step, BGRPO_TAG_SHARED, p.keys);
+#pragma unroll
+            for (int b = 0; b < FAN; ++b) {
+                float4 c;
+                if (WRITE) {
+                    float4 xi = noise4(e, gid_child0 + b, p.step, BGRPO_TAG_INNOV, p.keys);
+                    if (SHARED) {
+                        xi.x = fmaf(p.mix_innov, xi.x, p.mix_shared * xi0.x);
+                        xi.y = fmaf(p.mix_innov, xi.y, p.mix_shared * xi0.y);
+                        xi.z = fmaf(p.mix_innov, xi.z, p.mix_shared * xi0.z);
+                        xi.w = fmaf(p.mix_innov, xi.w, p.mix_shared * xi0.w);
+                    }
+                    c.x = fmaf(p.g, xi.x, m.x);
+                    c.y = fmaf(p.g, xi.y, m.y);
+                    c.z = fmaf(p.g, xi.z, m.z);
+                    c.w = fmaf(p.g, xi.w, m.w);
+                    zc[static_cast<size_t>(b) * D4 + e] = c;
+                } else {
+                    c = __ldcs(zc + static_cast<size_t>(b) * D4 + e);
+                }
+                const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
+                acc[b] = fmaf(dx, dx, acc[b]);
+                acc[b] = fmaf(dy, dy, acc[b]);
+                acc[b] = fmaf(dz, dz, acc[b]);
+                acc[b] = fmaf(dw, dw, acc[b]);
+            }
+        }
+    }
+}
+
 template <int FAN, bool SHARED, bool WRITE>
 __global__ void __launch_bounds__(kStreamThreads)
-step_kernel(const StepLaunch p) {
+step_kernel(const __grid_constant__ StepLaunch p) {
     const int chunk = blockIdx.x % p.nchunks;
     const int row = blockIdx.x / p.nchunks;             // tree * W_in + j
     const int tree = row / p.W_in;
     const int j = row - tree * p.W_in;
-    const int64_t D4 = p.D >> 2;
+    const uint32_t D4 = static_cast<uint32_t>(p.D >> 2);
     const int64_t tree_row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     const int parent = p.off_in + j;
     const int child0 = p.off_out + j * FAN;
@@ -123,62 +191,17 @@ step_kernel(const StepLaunch p) {
     float acc[FAN];
 #pragma unroll
     for (int b = 0; b < FAN; ++b) acc[b] = 0.0f;
+    const uint32_t e0 = static_cast<uint32_t>(chunk) * kChunkVec + threadIdx.x;
+    if (static_cast<uint32_t>(chunk + 1) * kChunkVec <= D4)
+        step_elements<FAN, SHARED, WRITE, true>(p, zp, xop, zc, e0, D4, gid_parent, gid_child0, streamed_operand, acc);
+    else
+        step_elements<FAN, SHARED, WRITE, false>(p, zp, xop, zc, e0, D4, gid_parent, gid_child0, streamed_operand, acc);
 
-    const int64_t e0 = static_cast<int64_t>(chunk) * kChunkVec + threadIdx.x;
-    float4 z[kVecPerThread], x[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int64_t e = e0 + k * kStreamThreads;
-        if (e < D4) {
-            z[k] = __ldcs(zp + e);                                   // read once: evict first
-            x[k] = streamed_operand ? __ldcs(xop + e) : __ldg(xop + e);   // the target mean is shared by the whole level
-        }
-    }
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int64_t e = e0 + k * kStreamThreads;
-        if (e < D4) {
-            float4 m;
-            m.x = fmaf(p.ca, z[k].x, p.cb * x[k].x);
-            m.y = fmaf(p.ca, z[k].y, p.cb * x[k].y);
-            m.z = fmaf(p.ca, z[k].z, p.cb * x[k].z);
-            m.w = fmaf(p.ca, z[k].w, p.cb * x[k].w);
-            float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (WRITE && SHARED) xi0 = noise4(static_cast<uint32_t>(e), gid_parent, p.step, BGRPO_TAG_SHARED, p.key0, p.key1);
-#pragma unroll
-            for (int b = 0; b < FAN; ++b) {
-                float4 c;
-                if (WRITE) {
-                    float4 xi = noise4(static_cast<uint32_t>(e), gid_child0 + b, p.step, BGRPO_TAG_INNOV, p.key0, p.key1);
-                    if (SHARED) {
-                        xi.x = fmaf(p.mix_innov, xi.x, p.mix_shared * xi0.x);
-                        xi.y = fmaf(p.mix_innov, xi.y, p.mix_shared * xi0.y);
-                        xi.z = fmaf(p.mix_innov, xi.z, p.mix_shared * xi0.z);
-                        xi.w = fmaf(p.mix_innov, xi.w, p.mix_shared * xi0.w);
-                    }
-                    c.x = fmaf(p.g, xi.x, m.x);
-                    c.y = fmaf(p.g, xi.y, m.y);
-                    c.z = fmaf(p.g, xi.z, m.z);
-                    c.w = fmaf(p.g, xi.w, m.w);
-                    zc[static_cast<int64_t>(b) * D4 + e] = c;
-                } else {
-                    c = __ldcs(zc + static_cast<int64_t>(b) * D4 + e);
-                }
-                const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
-                acc[b] = fmaf(dx, dx, acc[b]);
-                acc[b] = fmaf(dy, dy, acc[b]);
-                acc[b] = fmaf(dz, dz, acc[b]);
-                acc[b] = fmaf(dw, dw, acc[b]);
-            }
-        }
-    }
-
-    const bool last = publish_partials<FAN>(acc, p.partials, &p.counters[tree_row0 + parent], tree_row0 + child0, 1,
-                                            p.nchunks, chunk);
-    if (!last) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (warp < FAN) {
-        const int b = warp;
+    const bool last = publish_partials<FAN, true>(acc, p.partials, &p.counters[tree_row0 + parent], tree_row0 + child0, 1,
+                                                  p.nchunks, chunk);
+    if (!last) return;                                  // warps other than 0 always leave here
+    const int lane = threadIdx.x & 31;
+    for (int b = 0; b < FAN; ++b) {
         const double ss = row_total(p.partials, tree_row0 + child0 + b, 0, p.nchunks);
         if (lane == 0) {
             const int64_t r = tree_row0 + child0 + b;
@@ -201,7 +224,7 @@ step_kernel(const StepLaunch p) {
 // Leaf rewards: mode 0  r = -mean (z - target)^2 ; mode 1  r += scale * cos(z, target).
 template <int MODE>
 __global__ void __launch_bounds__(kStreamThreads)
-reward_kernel(const RewardLaunch p) {
+reward_kernel(const __grid_constant__ RewardLaunch p) {
     const int chunk = blockIdx.x % p.nchunks;
     const int row = blockIdx.x / p.nchunks;             // tree * leaves + l
     const int tree = row / p.leaves;
@@ -240,29 +263,27 @@ reward_kernel(const RewardLaunch p) {
             }
         }
     }
-    const bool last = publish_partials<NV>(acc, p.partials, &p.counters[node_row], node_row, NV, p.nchunks, chunk);
-    if (!last) return;
-    if ((threadIdx.x >> 5) == 0) {
-        if (MODE == 0) {
-            const double ss = row_total(p.partials, node_row, 0, p.nchunks);
-            if (threadIdx.x == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
-        } else {
-            const double dot = row_total(p.partials, node_row, 0, p.nchunks);
-            const double zz = row_total(p.partials, node_row, 1, p.nchunks);
-            const double tt = row_total(p.partials, node_row, 2, p.nchunks);
-            if (threadIdx.x == 0)
-                p.r[row] = static_cast<float>(static_cast<double>(p.r[row]) + static_cast<double>(p.scale) * dot / (sqrt(zz) * sqrt(tt)));
-        }
+    const bool last = publish_partials<NV, false>(acc, p.partials, &p.counters[node_row], node_row, NV, p.nchunks, chunk);
+    if (!last) return;                                  // only warp 0 of the row's last CTA goes on
+    if (MODE == 0) {
+        const double ss = row_total(p.partials, node_row, 0, p.nchunks);
+        if (threadIdx.x == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
+    } else {
+        const double dot = row_total(p.partials, node_row, 0, p.nchunks);
+        const double zz = row_total(p.partials, node_row, 1, p.nchunks);
+        const double tt = row_total(p.partials, node_row, 2, p.nchunks);
+        if (threadIdx.x == 0)
+            p.r[row] = static_cast<float>(static_cast<double>(p.r[row]) + static_cast<double>(p.scale) * dot / (sqrt(zz) * sqrt(tt)));
     }
 }
 
-__global__ void philox_words_kernel(uint32_t k0, uint32_t k1, uint32_t node, uint32_t step, uint32_t tag, uint4* out, int64_t nblk) {
+__global__ void philox_words_kernel(const __grid_constant__ PhiloxKeys keys, uint32_t node, uint32_t step, uint32_t tag, uint4* out, int64_t nblk) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i < nblk) out[i] = philox4x32_10(make_uint4(static_cast<uint32_t>(i), node, step, tag), k0, k1);
+    if (i < nblk) out[i] = philox4x32_10(make_uint4(static_cast<uint32_t>(i), node, step, tag), keys);
 }
-__global__ void philox_normals_kernel(uint32_t k0, uint32_t k1, uint32_t node, uint32_t step, uint32_t tag, float4* out, int64_t nblk) {
+__global__ void philox_normals_kernel(const __grid_constant__ PhiloxKeys keys, uint32_t node, uint32_t step, uint32_t tag, float4* out, int64_t nblk) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i < nblk) out[i] = noise4(static_cast<uint32_t>(i), node, step, tag, k0, k1);
+    if (i < nblk) out[i] = noise4(static_cast<uint32_t>(i), node, step, tag, keys);
 }
 
 template <int FAN>
@@ -280,7 +301,7 @@ cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s) {
     root_kernel<<<grid, kStreamThreads, 0, s>>>(t->buf.latents, t->buf.node_table, t->buf.logp, t->counters, t->status, t->D,
                                                 t->desc.n_trees, t->desc.nodes_cap, t->nchunks,
                                                 static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap),
-                                                static_cast<uint32_t>(t->desc.seed), static_cast<uint32_t>(t->desc.seed >> 32));
+                                                make_philox_keys(t->desc.seed));
     return cudaGetLastError();
 }
 
@@ -308,14 +329,14 @@ cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {
     if (nblk <= 0) return cudaSuccess;
     philox_words_kernel<<<static_cast<unsigned int>((nblk + 255) / 256), 256, 0, s>>>(
-        static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), node, step, tag, reinterpret_cast<uint4*>(out), nblk);
+        make_philox_keys(seed), node, step, tag, reinterpret_cast<uint4*>(out), nblk);
     return cudaGetLastError();
 }
 cudaError_t launch_philox_normals(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, float* out, int64_t n, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     const int64_t nblk = n / 4;
     philox_normals_kernel<<<static_cast<unsigned int>((nblk + 255) / 256), 256, 0, s>>>(
-        static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), node, step, tag, reinterpret_cast<float4*>(out), nblk);
+        make_philox_keys(seed), node, step, tag, reinterpret_cast<float4*>(out), nblk);
     return cudaGetLastError();
 }
 
