@@ -201,6 +201,30 @@ bgrpo_status bgrpo_philox_words_fill(uint64_t seed, uint32_t node_id, uint32_t s
 bgrpo_status bgrpo_philox_normal_fill(uint64_t seed, uint32_t node_id, uint32_t step, uint32_t tag, float* out_dev,
                                       int64_t n, void* stream);
 
+/* bgrpo_reward_mse_static - no counterpart in the paper; a deployment convenience.
+ * Some callers cannot give the library device scratch, because they cannot allocate device memory at the point where
+ * they call it: a serving or training process that handed all device memory to its own pool at start-up, a plug-in
+ * that runs inside another framework's step and must not trigger the device-wide synchronisation cudaMalloc implies,
+ * code under a fixed memory budget.  The tree handle of bgrpo_tree_init needs a caller-allocated scratch buffer, so
+ * those callers get this one self-contained call: r_out[i] = -mean_e (rows[i][e] - target[e])^2, the same reduction as
+ * bgrpo_leaf_reward_mse, with the reduction partials and ticket counters kept in a fixed BGRPO_STATIC_SCRATCH_BYTES
+ * array that is part of the library image (every GPU that loads the library holds that much until the process exits).
+ *   rows_dev   device [n_rows][D] float32, 16-byte aligned (e.g. the leaf rows of a latent pool)
+ *   target_dev device [D] float32, 16-byte aligned, shared by all rows
+ *   r_out_dev  device [n_rows] float32
+ * Limits: n_rows <= BGRPO_STATIC_MAX_ROWS and n_rows * ceil(D / 4096) <= (BGRPO_STATIC_SCRATCH_BYTES -
+ * 4 * BGRPO_STATIC_MAX_ROWS) / 8; anything larger returns BGRPO_ERR_CAPACITY and launches nothing (split the rows
+ * over several calls, one after the other).  D must be a positive multiple of 4 (INVALID_ARG otherwise).
+ * The call allocates and frees nothing.  The first call on each device looks up the array's device address (a host
+ * symbol lookup, done once per device with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: the call clears the counters
+ * it needs on `stream` before its kernel, but two calls that can overlap on the GPU (different streams without an
+ * ordering between them) race on it and give wrong results - keep calls stream-ordered. */
+#define BGRPO_STATIC_SCRATCH_BYTES (512 * 1024)
+#define BGRPO_STATIC_MAX_ROWS 1024
+bgrpo_status bgrpo_reward_mse_static(const float* rows_dev, const float* target_dev, int32_t n_rows, int64_t D,
+                                     float* r_out_dev, void* stream);
+
 void        bgrpo_tree_destroy(bgrpo_tree* tree);
 const char* bgrpo_status_string(bgrpo_status status);
 /* Last CUDA error text seen by this thread's most recent failing call ("" if none). */

@@ -77,6 +77,7 @@ _SIGNATURES = {
     "bgrpo_tree_sync_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "bgrpo_philox_words_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
     "bgrpo_philox_normal_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
+    "bgrpo_reward_mse_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_destroy": (None, [C.c_void_p]),
     "bgrpo_status_string": (C.c_char_p, [C.c_int]),
     "bgrpo_last_error": (C.c_char_p, []),
@@ -238,3 +239,14 @@ def philox_words_fill(seed, node_id, step, tag, out, n_blocks, stream=None):
 def philox_normal_fill(seed, node_id, step, tag, out, n, stream=None):
     _check(lib.bgrpo_philox_normal_fill(seed, node_id, step, tag, _ptr(out), n, _stream(stream)),
            "bgrpo_philox_normal_fill")
+
+
+STATIC_SCRATCH_BYTES, STATIC_MAX_ROWS = 512 * 1024, 1024
+
+
+def reward_mse_static(rows, target, n_rows: int, D: int, r_out, stream=None):
+    """-MSE of n_rows latent rows against one target, using the library's built-in scratch array instead of a
+    caller-allocated one (for callers that cannot allocate device memory when they call).  Raises BgrpoError
+    (ERR_CAPACITY) when n_rows or n_rows * ceil(D/4096) is beyond what the built-in array holds."""
+    _check(lib.bgrpo_reward_mse_static(_ptr(rows), _ptr(target), n_rows, D, _ptr(r_out), _stream(stream)),
+           "bgrpo_reward_mse_static")
