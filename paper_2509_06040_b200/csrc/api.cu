@@ -48,6 +48,7 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     size_t b = kScratchHeader;
     b += ((static_cast<size_t>(rows) * sizeof(unsigned int) + 255) / 256) * 256;
     b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
+    b += static_cast<size_t>(rows) * nchunks_of(D) * kStepWarps * sizeof(float);
     return b;
 }
 
@@ -78,6 +79,14 @@ void fill_coefficients(bgrpo_tree* t) {
 }
 
 bool tree_complete(const bgrpo_tree* t) { return t->depth == t->desc.T; }
+
+// Enqueues the small kernel that adds up a level's pending log-prob partials, if there are any.
+cudaError_t flush_pending(bgrpo_tree* t, cudaStream_t s) {
+    if (!t->pending.logp_out) return cudaSuccess;
+    const cudaError_t e = launch_finalize(t, t->pending, s);
+    t->pending.logp_out = nullptr;
+    return e;
+}
 
 }  // namespace
 
@@ -177,6 +186,8 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     t->status = reinterpret_cast<int32_t*>(sc);
     t->counters = reinterpret_cast<unsigned int*>(sc + kScratchHeader);
     t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
+    t->partialsf = reinterpret_cast<float*>(t->partials + rows * static_cast<size_t>(t->nchunks) * 3);
+    t->pending.logp_out = nullptr;
     fill_coefficients(t);
     st = bgrpo_tree_reset(t, desc->seed, stream);
     if (st != BGRPO_OK) {
@@ -190,6 +201,7 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
 bgrpo_status bgrpo_tree_reset(bgrpo_tree* t, uint64_t seed, void* stream) {
     if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
     t->desc.seed = seed;
+    t->pending.logp_out = nullptr;
     t->depth = 0;
     std::memset(&t->lv, 0, sizeof(t->lv));
     t->lv.width[0] = 1;
@@ -219,6 +231,9 @@ static void fill_step_launch(const bgrpo_tree* t, int step, const float* v_dev, 
     p->table = t->buf.node_table;
     p->partials = t->partials;
     p->counters = t->counters;
+    p->partialsf = t->partialsf;
+    p->status = t->status;
+    p->prev = t->pending;
     p->D = t->D;
     p->n_trees = t->desc.n_trees;
     p->nodes_cap = t->desc.nodes_cap;
@@ -257,6 +272,13 @@ bgrpo_status bgrpo_tree_step(bgrpo_tree* t, int32_t split_flag, const float* v_d
     p.logp_out = t->buf.logp;
     cudaError_t e = launch_step(p, as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "step kernel");
+    // this launch summed the previous level's log-probs in its prologue; its own are pending until the next
+    // launch, or until the flush below when the tree is complete
+    t->pending = FinalizeDesc{t->buf.logp, static_cast<int32_t>(W_out), static_cast<int32_t>(off_out), p.g, p.inv_2g2, p.logp_const};
+    if (i + 1 == t->desc.T) {
+        e = flush_pending(t, as_stream(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "log-prob flush kernel");
+    }
     t->lv.fanout[i] = fan;
     t->lv.width[i + 1] = static_cast<int32_t>(W_out);
     t->lv.offset[i + 2] = static_cast<int32_t>(off_out + W_out);
@@ -271,6 +293,10 @@ bgrpo_status bgrpo_tree_logprob(bgrpo_tree* t, int32_t step, const float* v_dev,
     if (!v_dev && !t->mu) return fail(BGRPO_ERR_STATE, "no velocity: pass v_dev or bind a linear velocity");
     if (v_dev && !aligned(v_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "v misaligned");
     const int first = step < 0 ? 0 : step, last = step < 0 ? t->depth - 1 : step;
+    {   // a step's own sums may still be pending and could live in the rows this call is about to rewrite
+        const cudaError_t e0 = flush_pending(t, as_stream(stream));
+        if (e0 != cudaSuccess) return cuda_fail(e0, "log-prob flush kernel");
+    }
     for (int i = first; i <= last; ++i) {
         StepLaunch p;
         fill_step_launch(t, i, v_dev, &p);
@@ -284,7 +310,10 @@ bgrpo_status bgrpo_tree_logprob(bgrpo_tree* t, int32_t step, const float* v_dev,
         p.logp_out = logp_out_dev;
         cudaError_t e = launch_step(p, as_stream(stream));
         if (e != cudaSuccess) return cuda_fail(e, "logprob kernel");
+        t->pending = FinalizeDesc{logp_out_dev, t->lv.width[i + 1], t->lv.offset[i + 1], p.g, p.inv_2g2, p.logp_const};
     }
+    const cudaError_t e = flush_pending(t, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "log-prob flush kernel");
     return BGRPO_OK;
 }
 
@@ -414,6 +443,7 @@ bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* t, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(t->status, 0, sizeof(word), as_stream(stream));
     if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (word & 2) return fail(BGRPO_ERR_CUDA, "a bounded wait inside the step kernel ran out");
     return (word & 1) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
 }
 

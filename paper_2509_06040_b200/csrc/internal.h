@@ -8,8 +8,22 @@
 
 namespace bgrpo {
 
-constexpr int kChunkVec = 1024;        // float4 per (parent, chunk) work item of the streaming kernels
-constexpr int kStreamThreads = 256;    // threads per CTA of the streaming kernels
+// Tile shape of the streaming kernels (overridable at build time for tuning sweeps).
+#ifndef BGRPO_STEP_THREADS
+#define BGRPO_STEP_THREADS 256
+#endif
+#ifndef BGRPO_STEP_VEC
+#define BGRPO_STEP_VEC 4
+#endif
+#ifndef BGRPO_STEP_STAGES
+#define BGRPO_STEP_STAGES 3
+#endif
+#ifndef BGRPO_STEP_CTAS
+#define BGRPO_STEP_CTAS 2
+#endif
+constexpr int kStreamThreads = BGRPO_STEP_THREADS;               // threads per CTA of the streaming kernels
+constexpr int kChunkVec = BGRPO_STEP_THREADS * BGRPO_STEP_VEC;   // float4 per (parent, chunk) work item
+constexpr int kStepWarps = kStreamThreads / 32;                  // log-prob partials per (row, chunk)
 constexpr int kScratchHeader = 256;    // bytes reserved at the start of scratch for the status word
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u;   // Philox4x32 multipliers and Weyl key increments (Salmon et al., SC'11)
@@ -46,6 +60,14 @@ struct StepCoef {
     float logp_const;    // -ln g - 0.5 ln(2 pi), 0 when g == 0
 };
 
+// Log-probs of a level whose per-(row, chunk, warp) partial sums are in scratch but not yet added up.  The sum is
+// taken by the next kernel the library enqueues on the stream (the next step's prologue, or a small flush kernel).
+struct FinalizeDesc {
+    float* logp_out;       // nullptr: nothing pending
+    int32_t W, off;        // rows off .. off+W-1 of every tree
+    float g, inv_2g2, logp_const;
+};
+
 struct LevelInfo {                       // layout of the tree grown so far
     int32_t width[BGRPO_MAX_T + 1];
     int32_t offset[BGRPO_MAX_T + 2];
@@ -70,7 +92,9 @@ struct bgrpo_tree {
     // scratch carving (device pointers inside buf.scratch)
     int32_t* status;
     unsigned int* counters;              // one ticket counter per (tree, node row)
-    double* partials;                    // [n_trees*nodes_cap][nchunks][3]
+    double* partials;                    // [n_trees*nodes_cap][nchunks][3]   (reward reductions)
+    float* partialsf;                    // [n_trees*nodes_cap][nchunks][kStepWarps] (log-prob sums of the step kernel)
+    bgrpo::FinalizeDesc pending;         // level whose log-probs still have to be summed
 };
 
 namespace bgrpo {
@@ -95,9 +119,13 @@ struct StepLaunch {
     int32_t shared_noise;      // 1: finite s at a split step
     int32_t write_children;    // 1: tree_step; 0: tree_logprob (children are read, nothing but logp is written)
     float* logp_out;           // destination of the log-probs (== logp for tree_step)
+    float* partialsf;          // [rows][nchunks][kStepWarps] warp sums of (z' - mean)^2
+    FinalizeDesc prev;         // level to finalize in this launch's prologue (logp_out == nullptr: none)
+    int32_t* status;           // device status word (bit 1: a bounded wait ran out)
 };
 cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s);
 cudaError_t launch_step(const StepLaunch& p, cudaStream_t s);
+cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStream_t s);
 
 struct RewardLaunch {
     const float* latents; const float* target; float* r; double* partials; unsigned int* counters;
