@@ -41,6 +41,7 @@ bgrpo_status check_desc(const bgrpo_tree_desc* d) {
 }
 
 int nchunks_of(int64_t D) { return static_cast<int>((D / 4 + kChunkVec - 1) / kChunkVec); }
+int nchunks_step_of(int64_t D) { return static_cast<int>((D / 4 + kStepChunkVec - 1) / kStepChunkVec); }
 
 size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     const int64_t rows = static_cast<int64_t>(d->n_trees) * d->nodes_cap;
@@ -48,7 +49,7 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     size_t b = kScratchHeader;
     b += ((static_cast<size_t>(rows) * sizeof(unsigned int) + 255) / 256) * 256;
     b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
-    b += static_cast<size_t>(rows) * nchunks_of(D) * kStepWarps * sizeof(float);
+    b += static_cast<size_t>(rows) * nchunks_step_of(D) * kStepWarps * sizeof(float);
     return b;
 }
 
@@ -170,6 +171,7 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     t->desc.t_grid = t->t_grid;
     t->D = static_cast<int64_t>(desc->tokens) * desc->channels;
     t->nchunks = nchunks_of(t->D);
+    t->nchunks_step = nchunks_step_of(t->D);
     t->independent = !(std::isfinite(desc->branch_corr_s) && desc->branch_corr_s >= 0.0f);
     if (t->independent) {
         t->mix_shared = 0.0f;
@@ -229,15 +231,12 @@ static void fill_step_launch(const bgrpo_tree* t, int step, const float* v_dev, 
     p->mu = v_dev ? nullptr : t->mu;
     p->logp = t->buf.logp;
     p->table = t->buf.node_table;
-    p->partials = t->partials;
-    p->counters = t->counters;
     p->partialsf = t->partialsf;
-    p->status = t->status;
     p->prev = t->pending;
     p->D = t->D;
     p->n_trees = t->desc.n_trees;
     p->nodes_cap = t->desc.nodes_cap;
-    p->nchunks = t->nchunks;
+    p->nchunks = t->nchunks_step;
     p->step = step;
     p->node_id_base = static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap);
     p->keys = make_philox_keys(t->desc.seed);
@@ -443,7 +442,6 @@ bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* t, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(t->status, 0, sizeof(word), as_stream(stream));
     if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "status read");
-    if (word & 2) return fail(BGRPO_ERR_CUDA, "a bounded wait inside the step kernel ran out");
     return (word & 1) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
 }
 

@@ -8,22 +8,17 @@
 
 namespace bgrpo {
 
-// Tile shape of the streaming kernels (overridable at build time for tuning sweeps).
-#ifndef BGRPO_STEP_THREADS
-#define BGRPO_STEP_THREADS 256
-#endif
-#ifndef BGRPO_STEP_VEC
-#define BGRPO_STEP_VEC 4
-#endif
-#ifndef BGRPO_STEP_STAGES
-#define BGRPO_STEP_STAGES 3
-#endif
-#ifndef BGRPO_STEP_CTAS
-#define BGRPO_STEP_CTAS 2
-#endif
-constexpr int kStreamThreads = BGRPO_STEP_THREADS;               // threads per CTA of the streaming kernels
-constexpr int kChunkVec = BGRPO_STEP_THREADS * BGRPO_STEP_VEC;   // float4 per (parent, chunk) work item
-constexpr int kStepWarps = kStreamThreads / 32;                  // log-prob partials per (row, chunk)
+constexpr int kStreamThreads = 256;    // threads per CTA of the root / reward kernels
+constexpr int kChunkVec = 1024;        // float4 per (row, chunk) work item of the root / reward kernels
+// Step kernel: 64-thread CTAs, 8 float4 per thread.  Measured on B200 against 128/256-thread CTAs, 2/4/6 float4 per
+// thread, persistent grids and a shared-memory ring fed by bulk asynchronous copies: the kernel is bound by
+// instruction issue (Philox + Box-Muller), and eight independent noise chains per thread with many small CTAs
+// per SM gave the best rate on both the 8 B/element and the 12 B/element workloads.
+constexpr int kStepThreads = 64;
+constexpr int kStepVec = 8;
+constexpr int kStepChunkVec = kStepThreads * kStepVec;   // 512 float4 = 8 KiB per operand tile
+constexpr int kStepWarps = kStepThreads / 32;            // log-prob partials per (row, chunk)
+constexpr int kStepCtasPerSm = 8;
 constexpr int kScratchHeader = 256;    // bytes reserved at the start of scratch for the status word
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u;   // Philox4x32 multipliers and Weyl key increments (Salmon et al., SC'11)
@@ -84,7 +79,8 @@ struct bgrpo_tree {
     bgrpo::LevelInfo lv;
     int32_t depth;                       // steps taken so far
     int64_t D;                           // elements per node
-    int32_t nchunks;                     // work items per node row
+    int32_t nchunks;                     // reward / root work items per node row
+    int32_t nchunks_step;                // step-kernel work items per node row
     bool independent;                    // s = inf: xi_b = eta_b
     float mix_shared, mix_innov;         // xi_b = mix_shared*xi_0 + mix_innov*eta_b
     const float* mu;                     // bound linear velocity (device), or nullptr
@@ -93,7 +89,7 @@ struct bgrpo_tree {
     int32_t* status;
     unsigned int* counters;              // one ticket counter per (tree, node row)
     double* partials;                    // [n_trees*nodes_cap][nchunks][3]   (reward reductions)
-    float* partialsf;                    // [n_trees*nodes_cap][nchunks][kStepWarps] (log-prob sums of the step kernel)
+    float* partialsf;                    // [n_trees*nodes_cap][nchunks_step][kStepWarps] (log-prob sums of the step kernel)
     bgrpo::FinalizeDesc pending;         // level whose log-probs still have to be summed
 };
 
@@ -106,10 +102,8 @@ struct StepLaunch {
     const float* mu;           // [n_trees][D] or nullptr
     float* logp;
     int32_t* table;            // SoA, stride = n_trees*nodes_cap
-    double* partials;
-    unsigned int* counters;
     int64_t D;                 // elements per row
-    int32_t n_trees, nodes_cap, nchunks;
+    int32_t n_trees, nodes_cap, nchunks;   // nchunks: step-kernel chunks per row
     int32_t W_in, off_in, off_out, fan, step, is_split;
     uint32_t node_id_base;     // tree_id_base * nodes_cap
     PhiloxKeys keys;
@@ -121,7 +115,6 @@ struct StepLaunch {
     float* logp_out;           // destination of the log-probs (== logp for tree_step)
     float* partialsf;          // [rows][nchunks][kStepWarps] warp sums of (z' - mean)^2
     FinalizeDesc prev;         // level to finalize in this launch's prologue (logp_out == nullptr: none)
-    int32_t* status;           // device status word (bit 1: a bounded wait ran out)
 };
 cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s);
 cudaError_t launch_step(const StepLaunch& p, cudaStream_t s);

@@ -3,13 +3,8 @@
 // and the leaf-reward reductions.  All of them are HBM-bound: every latent element is read or written once,
 // with 128-bit accesses, and the noise is generated in registers.
 //
-// Work decomposition: one CTA per (tree, parent node, chunk of kChunkVec float4).  A thread owns up to four
-// float4 of the parent row, loads them (and the velocity or target-mean operand) up front, evaluates the mean
-// once, and loops over the K children of the parent: the parent is read once however many children it has.
-// Sums over a row (log-prob, rewards) are float32 inside a thread's 16 elements (inside a warp's 512 for the
-// log-prob), double from there on: shared memory across warps, one double per (row, chunk) in scratch, and the
-// CTA that takes the last ticket of a row adds the chunk partials in a fixed order, so results do not depend
-// on scheduling.
+// Sums over a row are float32 inside a thread (inside a warp for the step's log-prob), double from there on, and
+// always added in a fixed order, so results do not depend on scheduling.
 #include "internal.h"
 #include "philox.cuh"
 
@@ -113,68 +108,22 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Fused step: a persistent, shared-memory-staged streaming kernel.
+// Fused step.  One CTA of kStepThreads threads per work item (tree, parent, chunk of kStepChunkVec float4).
 //
-// The grid holds kStepCtasPerSm CTAs per SM; CTA c owns the work items c, c + grid, c + 2 grid, ...  An item is
-// (tree, parent, chunk of kChunkVec float4).  One elected thread keeps kStages - 1 items ahead of the compute
-// threads with bulk asynchronous copies (cp.async.bulk, completion counted on an mbarrier) of the parent tile and
-// of the operand tile (velocity or target mean) into a ring of shared-memory stages, so DRAM latency is paid once
-// per CTA, not once per tile, and no register is tied up by loads in flight.  Every thread then reads its four
-// float4 of each tile from shared memory, releases the stage, evaluates the mean once and loops over the K
-// children (noise in registers, 128-bit stores).
+// A thread issues the 128-bit loads of its kStepVec float4 of the parent tile and of the operand tile (velocity or
+// target mean) first, then generates the noise of all its elements - Philox and Box-Muller depend on indices only,
+// so kStepVec independent chains per child are in flight while the loads travel - and only then touches the loaded
+// values: mean once per parent element, then for each of the K children z' = mean + g xi (128-bit store) and the
+// squared residual.  The parent is read once however many children it has.
 //
-// Log-prob: a warp adds its 512 squared residuals per child in float with a fixed shuffle tree and stores one
-// float per (child row, chunk, warp).  Nothing waits for those stores: the sums over chunks and warps are taken,
-// in double and in a fixed order, by the prologue of the NEXT launch on the stream (FinalizeDesc), or by the small
-// flush kernel when the tree is complete, so the hot loop has no fence, no atomic and no CTA-wide barrier.
+// Log-prob: a warp adds its squared residuals per child in float with a fixed shuffle tree and stores one float per
+// (child row, chunk, warp).  Nothing waits for those stores: the sums over chunks and warps are taken, in double and
+// in a fixed order, by the prologue of the NEXT launch on the stream (FinalizeDesc), or by the small flush kernel
+// when the tree is complete, so the kernel has no fence, no atomic and no CTA-wide barrier.
 //
 // FAN children per parent; SHARED: xi_b mixes a per-parent xi_0 (finite s at a split step); WRITE: true =
-// tree_step (draw noise, write children), false = tree_logprob (read children, score them).
-constexpr int kStages = BGRPO_STEP_STAGES;
-constexpr int kStepCtasPerSm = BGRPO_STEP_CTAS;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;              // bounded waits: after 2 s give up, flag, leave
-
-struct StepSmem {
-    float4 z[kStages][kChunkVec];
-    float4 x[kStages][kChunkVec];
-    unsigned long long full[kStages];
-    unsigned long long empty[kStages];
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Waits until the phase with the given parity has completed; false if the bounded spin ran out.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-    const uint32_t addr = smem_u32(bar);
-    unsigned long long t0 = 0;
-    for (;;) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-        unsigned long long now;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > kWaitLimitNs) return false;
-    }
-}
-// Bulk asynchronous copy global -> this CTA's shared memory; bytes % 16 == 0, both addresses 16-byte aligned.
-__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
+// tree_step (draw noise, write children), false = tree_logprob (read children, score them); FULL: the tile holds
+// kStepChunkVec float4, so no element needs a bounds test.
 
 // Adds up the pending level's partial sums: one warp per row, lanes stride over the row's nchunks * kStepWarps floats
 // in index order, then a fixed shuffle tree; double throughout.
@@ -197,176 +146,125 @@ __device__ __forceinline__ void finalize_rows(const FinalizeDesc& f, const float
     }
 }
 
-struct ItemAddr {
-    const float4* zp;       // parent tile
-    const float4* xop;      // operand tile
-    uint32_t vecs;          // float4 in this tile (kChunkVec, or fewer in a row's last chunk)
-};
-
-__device__ __forceinline__ void decode_item(const StepLaunch& p, int item, int& tree, int& j, int& chunk) {
-    chunk = item % p.nchunks;
-    const int row = item / p.nchunks;
-    tree = row / p.W_in;
-    j = row - tree * p.W_in;
+template <bool FULL>
+__device__ __forceinline__ void load_tile(const float4* __restrict__ zp, const float4* __restrict__ xop, bool streamed,
+                                          uint32_t vecs, float4 (&z)[kStepVec], float4 (&x)[kStepVec]) {
+#pragma unroll
+    for (int k = 0; k < kStepVec; ++k) {
+        const uint32_t t = threadIdx.x + k * kStepThreads;
+        if (FULL || t < vecs) {
+            z[k] = __ldcs(zp + t);                                   // read once: evict first
+            x[k] = streamed ? __ldcs(xop + t) : __ldg(xop + t);      // the target mean is shared by the whole level
+        }
+    }
 }
 
-__device__ __forceinline__ ItemAddr item_addr(const StepLaunch& p, int item) {
-    int tree, j, chunk;
-    decode_item(p, item, tree, j, chunk);
-    const int64_t D4 = p.D >> 2;
-    const int64_t e0 = static_cast<int64_t>(chunk) * kChunkVec;
-    ItemAddr a;
-    a.zp = reinterpret_cast<const float4*>(p.latents + (static_cast<int64_t>(tree) * p.nodes_cap + p.off_in + j) * p.D) + e0;
-    a.xop = (p.v ? reinterpret_cast<const float4*>(p.v + (static_cast<int64_t>(tree) * p.W_in + j) * p.D)
-                 : reinterpret_cast<const float4*>(p.mu + static_cast<int64_t>(tree) * p.D)) + e0;
-    a.vecs = static_cast<uint32_t>(min(static_cast<int64_t>(kChunkVec), D4 - e0));
-    return a;
+template <int FAN, bool SHARED, bool WRITE, bool FULL>
+__device__ __forceinline__ void compute_tile(const StepLaunch& p, const float4 (&z)[kStepVec], const float4 (&x)[kStepVec],
+                                             uint32_t vecs, uint32_t e_base, uint32_t D4, float4* zc, uint32_t gid_parent,
+                                             uint32_t gid_child0, float (&acc)[FAN]) {
+#pragma unroll
+    for (int k = 0; k < kStepVec; ++k) {
+        const uint32_t t = threadIdx.x + k * kStepThreads;
+        if (FULL || t < vecs) {
+            const uint32_t e = e_base + t;
+            float4 xi[FAN];
+            if (WRITE) {
+                float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (SHARED) xi0 = noise4(e, gid_parent, p.step, BGRPO_TAG_SHARED, p.keys);
+#pragma unroll
+                for (int b = 0; b < FAN; ++b) {
+                    xi[b] = noise4(e, gid_child0 + b, p.step, BGRPO_TAG_INNOV, p.keys);
+                    if (SHARED) {
+                        xi[b].x = fmaf(p.mix_innov, xi[b].x, p.mix_shared * xi0.x);
+                        xi[b].y = fmaf(p.mix_innov, xi[b].y, p.mix_shared * xi0.y);
+                        xi[b].z = fmaf(p.mix_innov, xi[b].z, p.mix_shared * xi0.z);
+                        xi[b].w = fmaf(p.mix_innov, xi[b].w, p.mix_shared * xi0.w);
+                    }
+                }
+            }
+            float4 m;
+            m.x = fmaf(p.ca, z[k].x, p.cb * x[k].x);
+            m.y = fmaf(p.ca, z[k].y, p.cb * x[k].y);
+            m.z = fmaf(p.ca, z[k].z, p.cb * x[k].z);
+            m.w = fmaf(p.ca, z[k].w, p.cb * x[k].w);
+#pragma unroll
+            for (int b = 0; b < FAN; ++b) {
+                float4 c;
+                if (WRITE) {
+                    c.x = fmaf(p.g, xi[b].x, m.x);
+                    c.y = fmaf(p.g, xi[b].y, m.y);
+                    c.z = fmaf(p.g, xi[b].z, m.z);
+                    c.w = fmaf(p.g, xi[b].w, m.w);
+                    zc[static_cast<size_t>(b) * D4 + e] = c;
+                } else {
+                    c = __ldcs(zc + static_cast<size_t>(b) * D4 + e);
+                }
+                const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
+                acc[b] = fmaf(dx, dx, acc[b]);
+                acc[b] = fmaf(dy, dy, acc[b]);
+                acc[b] = fmaf(dz, dz, acc[b]);
+                acc[b] = fmaf(dw, dw, acc[b]);
+            }
+        }
+    }
 }
 
 template <int FAN, bool SHARED, bool WRITE>
-__global__ void __launch_bounds__(kStreamThreads, kStepCtasPerSm)
-step_kernel(const __grid_constant__ StepLaunch p, int32_t n_items, int32_t* status) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    StepSmem& sm = *reinterpret_cast<StepSmem*>(smem_raw);
+__global__ void __launch_bounds__(kStepThreads, kStepCtasPerSm)
+step_kernel(const __grid_constant__ StepLaunch p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], kStepWarps);
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const int my_items = (n_items > static_cast<int>(blockIdx.x)) ? (n_items - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    // producer prologue: fill the ring
-    if (threadIdx.x == 0) {
-        for (int n = 0; n < kStages - 1 && n < my_items; ++n) {
-            const ItemAddr a = item_addr(p, blockIdx.x + n * gridDim.x);
-            mbar_expect_tx(&sm.full[n], 2 * a.vecs * static_cast<uint32_t>(sizeof(float4)));
-            bulk_load(sm.z[n], a.zp, a.vecs * static_cast<uint32_t>(sizeof(float4)), &sm.full[n]);
-            bulk_load(sm.x[n], a.xop, a.vecs * static_cast<uint32_t>(sizeof(float4)), &sm.full[n]);
-        }
-    }
-    // the previous level's log-probs, while the first tiles are on their way
+    // the previous level's log-probs (a handful of rows): summed by this launch
     if (p.prev.logp_out != nullptr)
         finalize_rows(p.prev, p.partialsf, p.n_trees, p.nodes_cap, p.nchunks, p.D, blockIdx.x * kStepWarps + warp, gridDim.x * kStepWarps);
 
+    const int chunk = blockIdx.x % p.nchunks;
+    const int row = blockIdx.x / p.nchunks;             // tree * W_in + j
+    const int tree = row / p.W_in;
+    const int j = row - tree * p.W_in;
     const uint32_t D4 = static_cast<uint32_t>(p.D >> 2);
-    bool ok = true;
-    for (int n = 0; n < my_items && ok; ++n) {
-        const int s = n % kStages;
-        const uint32_t parity = static_cast<uint32_t>(n / kStages) & 1u;
-        // producer: refill the stage that item n - 1 used (every warp released it when it began computing n - 1)
-        if (threadIdx.x == 0) {
-            const int m = n + kStages - 1;
-            if (m < my_items) {
-                const int sf = m % kStages;
-                if (m >= kStages) ok = mbar_wait(&sm.empty[sf], static_cast<uint32_t>(m / kStages - 1) & 1u);
-                if (ok) {
-                    const ItemAddr a = item_addr(p, blockIdx.x + m * gridDim.x);
-                    mbar_expect_tx(&sm.full[sf], 2 * a.vecs * static_cast<uint32_t>(sizeof(float4)));
-                    bulk_load(sm.z[sf], a.zp, a.vecs * static_cast<uint32_t>(sizeof(float4)), &sm.full[sf]);
-                    bulk_load(sm.x[sf], a.xop, a.vecs * static_cast<uint32_t>(sizeof(float4)), &sm.full[sf]);
-                }
-            }
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0 || warp != 0;      // warp 0 follows its lane 0
-        if (!ok) break;
-        if (!__all_sync(0xffffffffu, mbar_wait(&sm.full[s], parity) ? 1 : 0)) { ok = false; break; }   // warp-uniform
+    const uint32_t e_base = static_cast<uint32_t>(chunk) * kStepChunkVec;
+    const uint32_t vecs = min(static_cast<uint32_t>(kStepChunkVec), D4 - e_base);
+    const int64_t tree_row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    const int parent = p.off_in + j;
+    const int child0 = p.off_out + j * FAN;
+    const bool streamed = (p.v != nullptr);
+    const float4* __restrict__ zp = reinterpret_cast<const float4*>(p.latents + (tree_row0 + parent) * p.D) + e_base;
+    const float4* __restrict__ xop = (streamed ? reinterpret_cast<const float4*>(p.v + static_cast<int64_t>(row) * p.D)
+                                               : reinterpret_cast<const float4*>(p.mu + static_cast<int64_t>(tree) * p.D)) + e_base;
+    float4* zc = reinterpret_cast<float4*>(p.latents + (tree_row0 + child0) * p.D);
+    const uint32_t gid_parent = p.node_id_base + static_cast<uint32_t>(tree_row0 + parent);
+    const uint32_t gid_child0 = p.node_id_base + static_cast<uint32_t>(tree_row0 + child0);
 
-        int tree, j, chunk;
-        decode_item(p, blockIdx.x + n * gridDim.x, tree, j, chunk);
-        const uint32_t e_base = static_cast<uint32_t>(chunk) * kChunkVec;
-        const uint32_t vecs = min(static_cast<uint32_t>(kChunkVec), D4 - e_base);
-        float4 z[kVecPerThread], x[kVecPerThread];
+    float acc[FAN];
 #pragma unroll
-        for (int k = 0; k < kVecPerThread; ++k) {
-            const uint32_t t = threadIdx.x + k * kStreamThreads;
-            if (t < vecs) {
-                z[k] = sm.z[s][t];
-                x[k] = sm.x[s][t];
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[s]);           // this warp holds the tile in registers now
-
-        const int64_t tree_row0 = static_cast<int64_t>(tree) * p.nodes_cap;
-        const int parent = p.off_in + j;
-        const int child0 = p.off_out + j * FAN;
-        float4* zc = reinterpret_cast<float4*>(p.latents + (tree_row0 + child0) * p.D);
-        const uint32_t gid_parent = p.node_id_base + static_cast<uint32_t>(tree_row0 + parent);
-        const uint32_t gid_child0 = p.node_id_base + static_cast<uint32_t>(tree_row0 + child0);
-        float acc[FAN];
-#pragma unroll
-        for (int b = 0; b < FAN; ++b) acc[b] = 0.0f;
-#pragma unroll
-        for (int k = 0; k < kVecPerThread; ++k) {
-            const uint32_t t = threadIdx.x + k * kStreamThreads;
-            if (t < vecs) {
-                const uint32_t e = e_base + t;
-                float4 m;
-                m.x = fmaf(p.ca, z[k].x, p.cb * x[k].x);
-                m.y = fmaf(p.ca, z[k].y, p.cb * x[k].y);
-                m.z = fmaf(p.ca, z[k].z, p.cb * x[k].z);
-                m.w = fmaf(p.ca, z[k].w, p.cb * x[k].w);
-                float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (WRITE && SHARED) xi0 = noise4(e, gid_parent, p.step, BGRPO_TAG_SHARED, p.keys);
-#pragma unroll
-                for (int b = 0; b < FAN; ++b) {
-                    float4 c;
-                    if (WRITE) {
-                        float4 xi = noise4(e, gid_child0 + b, p.step, BGRPO_TAG_INNOV, p.keys);
-                        if (SHARED) {
-                            xi.x = fmaf(p.mix_innov, xi.x, p.mix_shared * xi0.x);
-                            xi.y = fmaf(p.mix_innov, xi.y, p.mix_shared * xi0.y);
-                            xi.z = fmaf(p.mix_innov, xi.z, p.mix_shared * xi0.z);
-                            xi.w = fmaf(p.mix_innov, xi.w, p.mix_shared * xi0.w);
-                        }
-                        c.x = fmaf(p.g, xi.x, m.x);
-                        c.y = fmaf(p.g, xi.y, m.y);
-                        c.z = fmaf(p.g, xi.z, m.z);
-                        c.w = fmaf(p.g, xi.w, m.w);
-                        zc[static_cast<size_t>(b) * D4 + e] = c;
-                    } else {
-                        c = __ldcs(zc + static_cast<size_t>(b) * D4 + e);
-                    }
-                    const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
-                    acc[b] = fmaf(dx, dx, acc[b]);
-                    acc[b] = fmaf(dy, dy, acc[b]);
-                    acc[b] = fmaf(dz, dz, acc[b]);
-                    acc[b] = fmaf(dw, dw, acc[b]);
-                }
-            }
-        }
-        // one float per (child row, chunk, warp); summed later in a fixed order
-#pragma unroll
-        for (int b = 0; b < FAN; ++b) {
-            float f = acc[b];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) f += __shfl_down_sync(0xffffffffu, f, o);
-            if (lane == 0)
-                p.partialsf[((tree_row0 + child0 + b) * p.nchunks + chunk) * kStepWarps + warp] = f;
-        }
-        if (WRITE && chunk == 0 && threadIdx.x < FAN) {      // node-table rows of the new children
-            const int b = threadIdx.x;
-            const int64_t rows = static_cast<int64_t>(p.n_trees) * p.nodes_cap;
-            const int64_t r = tree_row0 + child0 + b, rp = tree_row0 + parent;
-            p.table[r] = parent;
-            p.table[rows + r] = p.step + 1;
-            p.table[2 * rows + r] = p.is_split ? p.step : p.table[2 * rows + rp];
-            p.table[3 * rows + r] = p.is_split ? b : p.table[3 * rows + rp];
-        }
+    for (int b = 0; b < FAN; ++b) acc[b] = 0.0f;
+    float4 z[kStepVec], x[kStepVec];
+    if (vecs == kStepChunkVec) {
+        load_tile<true>(zp, xop, streamed, vecs, z, x);
+        compute_tile<FAN, SHARED, WRITE, true>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
+    } else {
+        load_tile<false>(zp, xop, streamed, vecs, z, x);
+        compute_tile<FAN, SHARED, WRITE, false>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
     }
-    if (!ok) {
-        // a bounded wait ran out (never expected): flag it, give copies already issued a bounded chance to land
-        // in this CTA's shared memory, and leave without touching anything else
-        if (lane == 0) atomicOr(status, 2);
-        if (threadIdx.x == 0)
-            for (int s = 0; s < kStages; ++s) (void)mbar_wait(&sm.full[s], 0);
+    // one float per (child row, chunk, warp); summed later in a fixed order
+#pragma unroll
+    for (int b = 0; b < FAN; ++b) {
+        float f = acc[b];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) f += __shfl_down_sync(0xffffffffu, f, o);
+        if (lane == 0)
+            p.partialsf[((tree_row0 + child0 + b) * p.nchunks + chunk) * kStepWarps + warp] = f;
     }
-    __syncthreads();      // the CTA's shared memory must stay allocated until every warp is done with it
+    if (WRITE && chunk == 0 && threadIdx.x < FAN) {      // node-table rows of the new children
+        const int b = threadIdx.x;
+        const int64_t rows = static_cast<int64_t>(p.n_trees) * p.nodes_cap;
+        const int64_t r = tree_row0 + child0 + b, rp = tree_row0 + parent;
+        p.table[r] = parent;
+        p.table[rows + r] = p.step + 1;
+        p.table[2 * rows + r] = p.is_split ? p.step : p.table[2 * rows + rp];
+        p.table[3 * rows + r] = p.is_split ? b : p.table[3 * rows + rp];
+    }
 }
 
 // Flush: adds up a pending level outside a step launch (the tree is complete, or tree_logprob is done).
@@ -442,39 +340,12 @@ __global__ void philox_normals_kernel(const __grid_constant__ PhiloxKeys keys, u
     if (i < nblk) out[i] = noise4(static_cast<uint32_t>(i), node, step, tag, keys);
 }
 
-int step_grid_limit() {
-    static int limit = 0;      // SM count of the current device (all devices of a node are alike)
-    if (limit == 0) {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            sms = 148;
-        limit = sms * kStepCtasPerSm;
-    }
-    return limit;
-}
-
-template <int FAN, bool SHARED, bool WRITE>
-cudaError_t launch_step_one(const StepLaunch& p, int32_t n_items, int32_t* status, cudaStream_t s) {
-    auto kernel = step_kernel<FAN, SHARED, WRITE>;
-    static bool configured[64] = {false};      // per kernel variant and device: the attribute belongs to both
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StepSmem)));
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
-    const int grid = n_items < step_grid_limit() ? n_items : step_grid_limit();
-    kernel<<<grid, kStreamThreads, sizeof(StepSmem), s>>>(p, n_items, status);
-    return cudaGetLastError();
-}
-
 template <int FAN>
-cudaError_t launch_step_fan(const StepLaunch& p, int32_t n_items, int32_t* status, cudaStream_t s) {
-    if (!p.write_children) return launch_step_one<FAN, false, false>(p, n_items, status, s);
-    if (p.shared_noise) return launch_step_one<FAN, true, true>(p, n_items, status, s);
-    return launch_step_one<FAN, false, true>(p, n_items, status, s);
+cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t s) {
+    if (!p.write_children) step_kernel<FAN, false, false><<<grid, kStepThreads, 0, s>>>(p);
+    else if (p.shared_noise) step_kernel<FAN, true, true><<<grid, kStepThreads, 0, s>>>(p);
+    else step_kernel<FAN, false, true><<<grid, kStepThreads, 0, s>>>(p);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -491,12 +362,12 @@ cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s) {
 cudaError_t launch_step(const StepLaunch& p, cudaStream_t s) {
     const int64_t items = static_cast<int64_t>(p.n_trees) * p.W_in * p.nchunks;
     if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    const int32_t n = static_cast<int32_t>(items);
+    const unsigned int grid = static_cast<unsigned int>(items);
     switch (p.fan) {
-        case 1: return launch_step_fan<1>(p, n, p.status, s);
-        case 2: return launch_step_fan<2>(p, n, p.status, s);
-        case 3: return launch_step_fan<3>(p, n, p.status, s);
-        case 4: return launch_step_fan<4>(p, n, p.status, s);
+        case 1: return launch_step_fan<1>(p, grid, s);
+        case 2: return launch_step_fan<2>(p, grid, s);
+        case 3: return launch_step_fan<3>(p, grid, s);
+        case 4: return launch_step_fan<4>(p, grid, s);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -504,7 +375,7 @@ cudaError_t launch_step(const StepLaunch& p, cudaStream_t s) {
 cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStream_t s) {
     const int rows = t->desc.n_trees * f.W;
     const int grid = (rows + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
-    finalize_kernel<<<grid < 1 ? 1 : grid, kStreamThreads, 0, s>>>(f, t->partialsf, t->desc.n_trees, t->desc.nodes_cap, t->nchunks, t->D);
+    finalize_kernel<<<grid < 1 ? 1 : grid, kStreamThreads, 0, s>>>(f, t->partialsf, t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D);
     return cudaGetLastError();
 }
 

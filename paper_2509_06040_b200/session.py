@@ -124,7 +124,7 @@ class TreeSession:
 
     def kernel_launches_per_pass(self) -> int:
         w = self.w
-        n = 1 + w.T * (2 if w.velocity == "mlp" else 1)           # root + (mlp +) step per depth
+        n = 1 + w.T * (2 if w.velocity == "mlp" else 1) + 1       # root + (mlp +) step per depth + log-prob flush
         n += 1 if w.reward in ("neg_mse_mu", "neg_mse_target", "normal_plus_cos") else 0
         n += 2                                                     # fuse+advantage, prune
         return n
