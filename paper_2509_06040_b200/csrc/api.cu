@@ -442,6 +442,7 @@ bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* t, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(t->status, 0, sizeof(word), as_stream(stream));
     if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (word & 4) return fail(BGRPO_ERR_CUDA, "a bounded wait inside the MLP velocity kernel ran out");
     return (word & 1) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
 }
 
@@ -478,7 +479,7 @@ bgrpo_status bgrpo_velocity_mlp(bgrpo_tree* t, const void* packed_dev, int32_t h
     const int i = t->depth;
     cudaError_t e = launch_mlp(t->buf.latents, static_cast<int64_t>(t->desc.nodes_cap) * t->D, static_cast<int64_t>(t->lv.offset[i]) * t->D,
                                t->desc.n_trees, static_cast<int64_t>(t->lv.width[i]) * t->desc.tokens, packed_dev, hidden,
-                               v_out_dev, as_stream(stream));
+                               v_out_dev, t->status, as_stream(stream));
     return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp kernel");
 }
 

@@ -146,6 +146,6 @@ cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s);
 size_t mlp_packed_bytes(int hidden);
 cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, void* packed, cudaStream_t s);
 cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
-                       const void* packed, int hidden, float* v_out, cudaStream_t s);
+                       const void* packed, int hidden, float* v_out, int32_t* status, cudaStream_t s);
 
 }  // namespace bgrpo

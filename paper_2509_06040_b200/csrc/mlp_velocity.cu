@@ -1,8 +1,398 @@
-// Per-token MLP velocity stage (placeholder until the tcgen05 kernel lands).
+// Per-token MLP velocity stage on the 5th-generation tensor cores (tcgen05 + tensor memory):
+//     v = bf16(GELU(bf16(z) W1)) W2,   z: [tokens][64] fp32,  W1: [64][H],  W2: [H][64],  fp32 accumulation, fp32 output.
+// It stands in for the denoiser mu_theta of Eq. 2 and is evaluated once per PARENT node of the frontier; the
+// K children of a parent share the result (the saving the rollout tree exists for).
+//
+// One persistent CTA per SM walks 128-token tiles.  For each tile the hidden dimension is cut into chunks of 128:
+//     GEMM1(c): D1[128 tok][128 hid]  = A[128 tok][64]      * W1_c        (4 MMAs of K = 16, accumulator in TMEM)
+//     GELU     : H_c = bf16(GELU(D1))   TMEM -> registers -> shared memory (the hidden activation never leaves the SM)
+//     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, accumulator in TMEM)
+// Warp roles: warp 0 streams the packed weight chunks (bulk asynchronous copies into a 3-stage ring), warp 1 owns
+// tensor memory and issues every MMA (one thread), warps 2..9 convert the latent tile to bf16, run the GELU epilogue
+// (two warps per TMEM lane quarter, 64 columns each) and write v.  D1 and H are double-buffered so GEMM1(c+1) and
+// the epilogue of chunk c overlap.  Operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the
+// MMA descriptors address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a
+// chunk (W1_c then W2_c, 32 KiB) arrives with a single copy.  No cluster multicast is used anywhere.
+//
+// Every wait is bounded (2 s): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
+// released and bit 2 of the status word is set.
 #include "internal.h"
 
 namespace bgrpo {
-size_t mlp_packed_bytes(int hidden) { return static_cast<size_t>(hidden) * 64 * 2 * 2; }
-cudaError_t launch_mlp_pack(const uint16_t*, const uint16_t*, int, void*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t launch_mlp(const float*, int64_t, int64_t, int, int64_t, const void*, int, float*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kTok = 128;                 // tokens per tile = MMA M
+constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
+constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
+constexpr int kWStages = 3;
+constexpr int kEpiWarps = 8;
+constexpr int kMlpThreads = (2 + kEpiWarps) * 32;
+constexpr uint32_t kChunkBytes = kHc * kCh * 2 * 2;      // W1_c (16 KiB) + W2_c (16 KiB)
+constexpr uint32_t kTmemCols = 512;       // D1: 2 x 128 columns, D2: 64 columns (power of two >= 320)
+constexpr uint32_t kD2Col = 256;
+constexpr unsigned long long kWaitNs = 2000000000ull;
+
+struct MlpSmem {
+    alignas(1024) unsigned char w[kWStages][kChunkBytes];   // per stage: W1_c tile [128 n][128 B], then W2_c as two [64 n][128 B] tiles
+    alignas(1024) unsigned char a[kTok * 128];              // bf16(z) tile [128 tok][128 B]
+    alignas(1024) unsigned char h[2][2][kTok * 128];        // [buffer][k half][128 tok][128 B]
+    unsigned long long w_full[kWStages], w_empty[kWStages];
+    unsigned long long a_full, a_empty, d1_full[2], d1_empty[2], h_full[2], h_empty[2], d2_full, d2_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase of the given parity; false after kWaitNs or once another thread has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort_flag) {
+    const uint32_t addr = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitNs) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// K-major operand tile of 128-byte rows, 128-byte swizzle: start address, leading offset 16 B (unused with swizzle),
+// stride between 8-row groups 1024 B, descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    return static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival when every MMA this thread has issued so far has completed.
+__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// GELU in its tanh form on the hardware tanh: 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).  It differs from the
+// erf form by < 5e-4 absolute, below the bf16 rounding of the activation that follows.
+__device__ __forceinline__ float gelu_fast(float x) {
+    const float x2 = x * x;
+    const float u = x * fmaf(x2, 0.0356774081f, 0.7978845608f);
+    float th;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(u));
+    const float hx = 0.5f * x;
+    return fmaf(hx, th, hx);
+}
+// byte offset of the 16-byte piece `c16` of row r inside a 128-byte-swizzled tile of 128-byte rows
+__device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c16) { return r * 128u + ((c16 ^ (r & 7u)) << 4); }
+
+struct MlpArgs {
+    const float* latents;     // pool base
+    int64_t tree_stride;      // elements between trees in the pool
+    int64_t row_offset;       // elements from a tree's base to its frontier
+    int64_t tokens_per_tree;  // frontier tokens of one tree (W_i * tokens)
+    int64_t n_tokens;         // all frontier tokens
+    const unsigned char* packed;
+    float* v_out;
+    int32_t n_chunks;         // hidden / 128
+    int32_t n_tiles;
+    int32_t* status;
+};
+
+__global__ void __launch_bounds__(kMlpThreads, 1)
+mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // the swizzled operand tiles need 1024-byte alignment; the launch reserves 1 KiB of slack for this round-up
+    MlpSmem& sm = *reinterpret_cast<MlpSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort_flag = &sm.abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWStages; ++s) { mbar_init(&sm.w_full[s], 1); mbar_init(&sm.w_empty[s], 1); }
+        mbar_init(&sm.a_full, kEpiWarps);
+        mbar_init(&sm.a_empty, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.d1_full[b], 1);
+            mbar_init(&sm.d1_empty[b], kEpiWarps);
+            mbar_init(&sm.h_full[b], kEpiWarps);
+            mbar_init(&sm.h_empty[b], 1);
+        }
+        mbar_init(&sm.d2_full, 1);
+        mbar_init(&sm.d2_empty, kEpiWarps);
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {      // tensor memory: this warp allocates and, at the end, frees
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const int n_my_tiles = (p.n_tiles > static_cast<int>(blockIdx.x)) ? (p.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    const int NC = p.n_chunks;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- weight producer
+        if (lane == 0) {
+            int g = 0;      // running chunk count across tiles
+            for (int it = 0; it < n_my_tiles && !*abort_flag; ++it) {
+                for (int c = 0; c < NC; ++c, ++g) {
+                    const int s = g % kWStages;
+                    if (g >= kWStages && !mbar_wait(&sm.w_empty[s], static_cast<uint32_t>(g / kWStages - 1) & 1u, abort_flag)) break;
+                    mbar_expect_tx(&sm.w_full[s], kChunkBytes);
+                    bulk_load(sm.w[s], p.packed + static_cast<size_t>(c) * kChunkBytes, kChunkBytes, &sm.w_full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc1 = umma_idesc(kTok, kHc), idesc2 = umma_idesc(kTok, kCh);
+            const uint64_t a_desc = umma_desc(smem_u32(sm.a));
+            int g = 0;
+            bool ok = true;
+            // GEMM1 of chunk c of the current tile (global chunk index gc): D1[gc % 2] = A * W1_c
+            auto gemm1 = [&](int gc) -> bool {
+                const int s = gc % kWStages, b = gc & 1;
+                if (!mbar_wait(&sm.w_full[s], static_cast<uint32_t>(gc / kWStages) & 1u, abort_flag)) return false;
+                if (gc >= 2 && !mbar_wait(&sm.d1_empty[b], static_cast<uint32_t>(gc / 2 - 1) & 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint64_t b_desc = umma_desc(smem_u32(sm.w[s]));
+#pragma unroll
+                for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
+                    umma_bf16(tmem + static_cast<uint32_t>(b) * kHc, a_desc + 2u * k, b_desc + 2u * k, idesc1, k > 0 ? 1u : 0u);
+                umma_commit(&sm.d1_full[b]);
+                return true;
+            };
+            for (int it = 0; it < n_my_tiles && ok; ++it) {
+                ok = mbar_wait(&sm.a_full, static_cast<uint32_t>(it) & 1u, abort_flag);
+                if (ok) ok = gemm1(g);
+                for (int c = 0; c < NC && ok; ++c) {
+                    const int gc = g + c;
+                    if (c + 1 < NC) {
+                        ok = gemm1(gc + 1);
+                        if (!ok) break;
+                    } else {
+                        umma_commit(&sm.a_empty);          // every GEMM1 of this tile has been issued
+                    }
+                    const int s = gc % kWStages, b = gc & 1;
+                    ok = mbar_wait(&sm.h_full[b], static_cast<uint32_t>(gc / 2) & 1u, abort_flag);
+                    if (ok && c == 0 && it > 0) ok = mbar_wait(&sm.d2_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < kHc / 16; ++k) {
+                        const uint64_t ha = umma_desc(smem_u32(sm.h[b][k / 4])) + 2u * (k % 4);
+                        const uint64_t wb = umma_desc(smem_u32(sm.w[s] + kHc * 128 + (k / 4) * (kCh * 128))) + 2u * (k % 4);
+                        umma_bf16(tmem + kD2Col, ha, wb, idesc2, (c > 0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&sm.h_empty[b]);
+                    umma_commit(&sm.w_empty[s]);
+                    if (c == NC - 1) umma_commit(&sm.d2_full);
+                }
+                g += NC;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int ew = warp - 2;                  // 0..7
+        const uint32_t quarter = static_cast<uint32_t>(warp & 3);   // TMEM lanes this warp may touch: 32*quarter .. +31
+        const uint32_t half = static_cast<uint32_t>(ew >> 2);       // which 64 of the chunk's 128 columns
+        const uint32_t row = quarter * 32u + static_cast<uint32_t>(lane);       // token row of this thread in the tile
+        const uint32_t lane_addr = (quarter * 32u) << 16;
+        bool ok = true;
+        int g = 0;
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
+            // ---- latent tile -> bf16, K-major swizzled.  A warp covers 2 rows per pass (16 lanes x 16 B per row).
+            if (it > 0) ok = mbar_wait(&sm.a_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;      // keep every verdict warp-uniform: the TMEM loads are warp-wide
+            if (!ok) break;
+            for (int pass = 0; pass < kTok / (2 * kEpiWarps); ++pass) {
+                const uint32_t r = static_cast<uint32_t>(pass * 2 * kEpiWarps + ew * 2 + (lane >> 4));
+                const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row
+                const int64_t q = tok0 + r;
+                float4 zv = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q < p.n_tokens) {
+                    const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
+                    zv = __ldcs(reinterpret_cast<const float4*>(p.latents + tree * p.tree_stride + p.row_offset + rr * kCh) + c4);
+                }
+                uint2 packed2;
+                packed2.x = pack_bf16(zv.x, zv.y);
+                packed2.y = pack_bf16(zv.z, zv.w);
+                *reinterpret_cast<uint2*>(sm.a + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
+            }
+            proxy_fence();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.a_full);
+
+            for (int c = 0; c < NC && ok; ++c) {
+                const int gc = g + c, b = gc & 1;
+                ok = mbar_wait(&sm.d1_full[b], static_cast<uint32_t>(gc / 2) & 1u, abort_flag);
+                if (ok && gc >= 2) ok = mbar_wait(&sm.h_empty[b], static_cast<uint32_t>(gc / 2 - 1) & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int grp = 0; grp < 2; ++grp) {          // 2 x 32 columns of this warp's 64
+                    uint32_t acc[32];
+                    const uint32_t col = static_cast<uint32_t>(b) * kHc + half * 64u + static_cast<uint32_t>(grp) * 32u;
+                    tmem_ld32(tmem + lane_addr + col, acc);
+                    tmem_ld_wait();
+                    unsigned char* htile = sm.h[b][half];     // hidden columns half*64 .. +63 are K half `half` of GEMM2
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {             // 8 columns -> one 16-byte piece
+                        uint4 piece;
+                        piece.x = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 0])), gelu_fast(__uint_as_float(acc[8 * j + 1])));
+                        piece.y = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 2])), gelu_fast(__uint_as_float(acc[8 * j + 3])));
+                        piece.z = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 4])), gelu_fast(__uint_as_float(acc[8 * j + 5])));
+                        piece.w = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 6])), gelu_fast(__uint_as_float(acc[8 * j + 7])));
+                        *reinterpret_cast<uint4*>(htile + sw128(row, static_cast<uint32_t>(grp * 4 + j))) = piece;
+                    }
+                }
+                tc_fence_before();
+                proxy_fence();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&sm.d1_empty[b]);
+                    mbar_arrive(&sm.h_full[b]);
+                }
+            }
+            if (!ok) break;
+            g += NC;
+            // ---- output tile: D2 -> v (this warp's 32 of the 64 channels)
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d2_full, static_cast<uint32_t>(it) & 1u, abort_flag) ? 1 : 0) != 0;
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t out[32];
+            tmem_ld32(tmem + lane_addr + kD2Col + half * 32u, out);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.d2_empty);
+            const int64_t q = tok0 + row;
+            if (q < p.n_tokens) {
+                float4* dst = reinterpret_cast<float4*>(p.v_out + q * kCh + half * 32u);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(out[4 * j]), __uint_as_float(out[4 * j + 1]), __uint_as_float(out[4 * j + 2]),
+                                         __uint_as_float(out[4 * j + 3]));
+            }
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+    if (threadIdx.x == 0 && sm.abort_flag) atomicOr(p.status, 4);
+}
+
+// Reorders W1 [64][H] and W2 [H][64] (bf16 bits) into per-chunk shared-memory images: for chunk c,
+//   bytes [0, 16 KiB):      W1_c as [128 n = hidden][64 k = channel], 128-byte rows, 128-byte swizzle
+//   bytes [16 KiB, 32 KiB): W2_c as two tiles [64 n = channel][64 k = hidden], one per half of the chunk's hidden range
+__global__ void mlp_pack_kernel(const uint16_t* __restrict__ W1, const uint16_t* __restrict__ W2, int hidden, unsigned char* __restrict__ packed) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;      // one bf16 element of W1 and one of W2 per thread
+    if (idx >= hidden * kCh) return;
+    {   // W1[k][j]
+        const int k = idx / hidden, j = idx - k * hidden;
+        const int c = j / kHc, n = j - c * kHc;
+        const uint32_t off = static_cast<uint32_t>(n) * 128u + (((static_cast<uint32_t>(k) >> 3) ^ (static_cast<uint32_t>(n) & 7u)) << 4) + (static_cast<uint32_t>(k) & 7u) * 2u;
+        *reinterpret_cast<uint16_t*>(packed + static_cast<size_t>(c) * kChunkBytes + off) = W1[idx];
+    }
+    {   // W2[j][n]
+        const int j = idx / kCh, n = idx - j * kCh;
+        const int c = j / kHc, jj = j - c * kHc, hf = jj / 64, kk = jj - hf * 64;
+        const uint32_t off = static_cast<uint32_t>(n) * 128u + (((static_cast<uint32_t>(kk) >> 3) ^ (static_cast<uint32_t>(n) & 7u)) << 4) + (static_cast<uint32_t>(kk) & 7u) * 2u;
+        *reinterpret_cast<uint16_t*>(packed + static_cast<size_t>(c) * kChunkBytes + kHc * 128 + hf * (kCh * 128) + off) = W2[idx];
+    }
+}
+
+}  // namespace
+
+size_t mlp_packed_bytes(int hidden) { return static_cast<size_t>(hidden / kHc) * kChunkBytes; }
+
+cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, void* packed, cudaStream_t s) {
+    const int n = hidden * kCh;
+    mlp_pack_kernel<<<(n + 255) / 256, 256, 0, s>>>(W1, W2, hidden, static_cast<unsigned char*>(packed));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
+                       const void* packed, int hidden, float* v_out, int32_t* status, cudaStream_t s) {
+    static bool configured[64] = {false};
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(mlp_velocity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(MlpSmem) + 1024));
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    MlpArgs a;
+    a.latents = latents;
+    a.tree_stride = tree_stride;
+    a.row_offset = row_offset;
+    a.tokens_per_tree = tokens_per_tree;
+    a.n_tokens = static_cast<int64_t>(n_trees) * tokens_per_tree;
+    a.packed = static_cast<const unsigned char*>(packed);
+    a.v_out = v_out;
+    a.n_chunks = hidden / kHc;
+    const int64_t tiles = (a.n_tokens + kTok - 1) / kTok;
+    if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    a.n_tiles = static_cast<int32_t>(tiles);
+    a.status = status;
+    const int grid = a.n_tiles < sms ? a.n_tiles : sms;
+    mlp_velocity_kernel<<<grid, kMlpThreads, sizeof(MlpSmem) + 1024, s>>>(a);
+    return cudaGetLastError();
+}
+
 }  // namespace bgrpo

@@ -1,0 +1,111 @@
+"""The tcgen05 MLP velocity stage against the oracle's bf16-emulating MLP, stage by stage: at every depth the
+oracle's frontier latents are written into the device pool (so both sides see the same z), the CUDA stage runs
+through the C ABI, and its output is compared under  |d| <= 2e-2 |v| + 2e-2 rms(v)  (bf16 operands; the CUDA side
+uses the tanh form of GELU and fp32 accumulation).  The tree is then advanced with the oracle's velocity, so
+later depths exercise frontiers of several nodes, several trees and ragged 128-token tiles."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mlp, sde
+from oracle import tree as otree
+from workloads import Workload, make_inputs
+
+from test_gpu_parity import B, LATENT_TOL, f32  # noqa: F401
+
+pytestmark = pytest.mark.gpu
+
+
+def _mlp_close(got, ref):
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    return np.all(np.abs(got - ref) <= 2e-2 * np.abs(ref) + 2e-2 * rms), float(np.abs(got - ref).max()), rms
+
+
+@pytest.mark.parametrize("tokens,hidden,n_trees,K,splits", [(200, 256, 2, 2, (0, 2)), (37, 128, 3, 3, (1,)), (512, 3072, 1, 2, (0, 1))])
+def test_mlp_stage_matches_oracle_at_every_depth(B, tokens, hidden, n_trees, K, splits):
+    from paper_2509_06040_b200.session import TreeSession
+    w = Workload(name="mlp", n_trees=n_trees, tokens=tokens, channels=64, T=3, K=K, splits=splits, sigma=0.3,
+                 velocity="mlp", reward="mixture", hidden=hidden)
+    inp = make_inputs(w)
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    v_store = {}
+
+    def vel_factory(t):
+        def vel(z, i, p):
+            v = mlp.mlp_velocity(z.reshape(w.tokens, w.channels), inp.W1, inp.W2).reshape(-1)
+            v_store[(t, i, p)] = v
+            return v
+        return vel
+
+    lats = [sde.rollout(topo, w.D, grid, f32(w.sigma), w.branch_corr_s, w.seed, vel_factory(t), tree_id=t, nodes_cap=topo.nodes)[0]
+            for t in range(n_trees)]
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+    s.init()
+    worst = 0.0
+    for i in range(w.T):
+        level = list(topo.level(i))
+        for t in range(n_trees):       # same z on both sides: the oracle's frontier goes into the pool
+            s.latents[t, level[0]:level[-1] + 1].copy_(torch.from_numpy(lats[t][level[0]:level[-1] + 1]))
+        s.v.fill_(float("nan"))
+        B.velocity_mlp(s.tree, s.packed, w.hidden, s.v)
+        torch.cuda.synchronize()
+        B.tree_sync_status(s.tree)
+        ref = np.stack([np.stack([v_store[(t, i, p)] for p in level]) for t in range(n_trees)])
+        got = s.v.cpu().numpy().reshape(-1)[:ref.size].reshape(ref.shape)
+        ok, err, rms = _mlp_close(got, ref)
+        assert ok, (i, err, rms)
+        worst = max(worst, err / rms)
+        B.tree_step(s.tree, 1 if i in w.splits else 0, torch.from_numpy(ref).cuda())
+    torch.cuda.synchronize()
+    assert worst < 2e-2
+    # the teacher-forced steps reproduce the oracle's latents
+    for t in range(n_trees):
+        assert np.abs(s.latents[t].cpu().numpy() - lats[t]).max() <= LATENT_TOL
+
+
+def test_mlp_special_weights(B):
+    """Zero weights give v = 0; W1 = [I, -I], W2 = [I; -I] gives v = GELU(z) - GELU(-z) = z up to bf16 rounding."""
+    from paper_2509_06040_b200.session import TreeSession
+    from workloads import Inputs
+    w = Workload(name="mlp_id", n_trees=1, tokens=130, channels=64, T=1, K=1, splits=(), sigma=0.3,
+                 velocity="mlp", reward="mixture", hidden=128)
+    W1 = np.concatenate([np.eye(64), -np.eye(64)], axis=1).astype(np.float32)
+    W2 = np.concatenate([np.eye(64), -np.eye(64)], axis=0).astype(np.float32)
+    for scale in (1.0, 0.0):
+        s = TreeSession(w)
+        s.upload_inputs(Inputs(W1=W1 * scale, W2=W2 * scale))
+        s.init()
+        B.velocity_mlp(s.tree, s.packed, w.hidden, s.v)
+        torch.cuda.synchronize()
+        z = s.latents[0, 0].cpu().numpy().reshape(130, 64)
+        v = s.v.cpu().numpy().reshape(-1)[:130 * 64].reshape(130, 64)
+        if scale == 0.0:
+            assert np.all(v == 0.0)
+        else:
+            assert np.allclose(v, z, rtol=2 ** -6, atol=4e-3)
+
+
+def test_full_mlp_rollout_stays_close_to_the_oracle(B):
+    """End to end with the CUDA MLP feeding the CUDA step: drift against the all-oracle rollout is reported, and
+    bounded loosely (the 1e-5 latent tolerance cannot hold downstream of a bf16 stage)."""
+    from paper_2509_06040_b200.session import TreeSession
+    w = Workload(name="mlp_e2e", n_trees=1, tokens=256, channels=64, T=6, K=2, splits=(0, 3), sigma=0.3,
+                 velocity="mlp", reward="mixture", hidden=512)
+    inp = make_inputs(w)
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    lat, logp = sde.rollout(topo, w.D, grid, f32(w.sigma), math.inf, w.seed,
+                            lambda z, i, p: mlp.mlp_velocity(z.reshape(w.tokens, 64), inp.W1, inp.W2).reshape(-1))
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+    s.rollout()
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    drift = np.abs(s.latents[0].cpu().numpy() - lat).max()
+    print("max latent drift through the bf16 stage:", drift)
+    assert drift < 5e-3
+    assert np.abs(s.logp[0].cpu().numpy() - logp).max() < 1e-3
