@@ -7,12 +7,16 @@
 //     GEMM1(c): D1[128 tok][128 hid]  = A[128 tok][64]      * W1_c        (4 MMAs of K = 16, accumulator in TMEM)
 //     GELU     : H_c = bf16(GELU(D1))   TMEM -> registers -> shared memory (the hidden activation never leaves the SM)
 //     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, accumulator in TMEM)
-// Warp roles: warp 0 streams the packed weight chunks (bulk asynchronous copies into a 3-stage ring), warp 1 owns
-// tensor memory and issues every MMA (one thread), warps 2..9 convert the latent tile to bf16, run the GELU epilogue
-// (two warps per TMEM lane quarter, 64 columns each) and write v.  D1 and H are double-buffered so GEMM1(c+1) and
-// the epilogue of chunk c overlap.  Operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the
-// MMA descriptors address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a
-// chunk (W1_c then W2_c, 32 KiB) arrives with a single copy.  No cluster multicast is used anywhere.
+// Warp roles:
+//     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 4-stage ring of W1 chunks,
+//                  lane 1 a 3-stage ring of W2 chunks (W1_c is needed two chunks earlier than W2_c);
+//     warp 1       owns tensor memory and issues every MMA from one thread; GEMM1 runs two chunks ahead (D1 is
+//                  triple-buffered), GEMM2(c) overlaps the epilogue of chunk c + 1 (H is double-buffered);
+//     warps 2..17  GELU epilogue, four warps per TMEM lane quarter with 32 columns each, and the output tile;
+//     warp 18      converts the NEXT tile's latents to bf16 into the second A buffer while the current tile computes.
+// Operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors address; the
+// weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with one copy
+// per matrix.  No cluster multicast is used anywhere.
 //
 // Every wait is bounded (2 s): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
 // released and bit 2 of the status word is set.
@@ -24,22 +28,39 @@ namespace {
 constexpr int kTok = 128;                 // tokens per tile = MMA M
 constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
 constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
-constexpr int kWStages = 3;
-constexpr int kEpiWarps = 8;
-constexpr int kMlpThreads = (2 + kEpiWarps) * 32;
-constexpr uint32_t kChunkBytes = kHc * kCh * 2 * 2;      // W1_c (16 KiB) + W2_c (16 KiB)
-constexpr uint32_t kTmemCols = 512;       // D1: 2 x 128 columns, D2: 64 columns (power of two >= 320)
-constexpr uint32_t kD2Col = 256;
+constexpr int kW1Stages = 4;
+constexpr int kW2Stages = 3;
+constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 32 columns of a chunk each
+constexpr int kLoaderWarp = 2 + kEpiWarps;
+constexpr int kMlpThreads = (3 + kEpiWarps) * 32;
+constexpr uint32_t kTileBytes = kTok * 128;              // one [128 rows][128 B] operand tile = 16 KiB
+constexpr uint32_t kChunkBytes = 2 * kTileBytes;         // packed weights of a chunk: W1_c (16 KiB) then W2_c (16 KiB)
+constexpr int kD1Bufs = 3;                // GEMM1 runs two chunks ahead of the epilogue
+constexpr uint32_t kTmemCols = 512;       // D1: 3 x 128 columns, D2: 64 columns (power of two >= 448)
+constexpr uint32_t kD2Col = kD1Bufs * kHc;
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 struct MlpSmem {
-    alignas(1024) unsigned char w[kWStages][kChunkBytes];   // per stage: W1_c tile [128 n][128 B], then W2_c as two [64 n][128 B] tiles
-    alignas(1024) unsigned char a[kTok * 128];              // bf16(z) tile [128 tok][128 B]
-    alignas(1024) unsigned char h[2][2][kTok * 128];        // [buffer][k half][128 tok][128 B]
-    unsigned long long w_full[kWStages], w_empty[kWStages];
-    unsigned long long a_full, a_empty, d1_full[2], d1_empty[2], h_full[2], h_empty[2], d2_full, d2_empty;
+    alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
+    alignas(1024) unsigned char w2[kW2Stages][kTileBytes];  // W2_c as two [64 n = channel][128 B = 64 hidden] tiles
+    alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
+    alignas(1024) unsigned char h[2][2][kTileBytes];        // [buffer][k half][128 tok][128 B]
+    unsigned long long w1_full[kW1Stages], w1_empty[kW1Stages], w2_full[kW2Stages], w2_empty[kW2Stages];
+    unsigned long long a_full[2], a_empty[2], d1_full[kD1Bufs], d1_empty[kD1Bufs], h_full[2], h_empty[2], d2_full, d2_empty;
     uint32_t tmem_base;
     int abort_flag;
+};
+
+// Position in a ring of N slots: slot index, phase parity of the slot's current use, and whether the ring has
+// wrapped yet (before that, "slot is free" needs no wait).
+template <int N>
+struct Ring {
+    int slot = 0;
+    uint32_t phase = 0;
+    bool wrapped = false;
+    __device__ __forceinline__ void advance() {
+        if (++slot == N) { slot = 0; phase ^= 1u; wrapped = true; }
+    }
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -55,6 +76,15 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t
 // Bounded wait for the phase of the given parity; false after kWaitNs or once another thread has raised the abort flag.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort_flag) {
     const uint32_t addr = smem_u32(bar);
+    {   // common case: the phase is already complete, or completes within the hardware's own suspend window
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
     unsigned long long t0 = 0;
     for (;;) {
         uint32_t done;
@@ -76,11 +106,13 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                  ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// K-major operand tile of 128-byte rows, 128-byte swizzle: start address, leading offset 16 B (unused with swizzle),
-// stride between 8-row groups 1024 B, descriptor version 1, layout type 2 (128-byte swizzle).
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-    return static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
+// Shared-memory operand descriptor of a K-major tile of 128-byte rows in the 128-byte-swizzle layout: start address
+// >> 4 in bits 0-13, leading offset 16 B (unused with swizzle) in bits 16-29, stride between 8-row groups (1024 B) >> 4
+// in bits 32-45, descriptor version 1 in bits 46-47, layout type 2 (128-byte swizzle) in bits 61-63.
+// Split in words: only the low word depends on the address, and advancing by n bytes adds n >> 4.
+constexpr uint32_t kDescHi = 64u | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(const void* smem_ptr) { return ((smem_u32(smem_ptr) >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return (static_cast<uint64_t>(kDescHi) << 32) | lo; }
 // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
 __host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
@@ -103,6 +135,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
           "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -150,14 +189,17 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     volatile int* abort_flag = &sm.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kWStages; ++s) { mbar_init(&sm.w_full[s], 1); mbar_init(&sm.w_empty[s], 1); }
-        mbar_init(&sm.a_full, kEpiWarps);
-        mbar_init(&sm.a_empty, 1);
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&sm.d1_full[b], 1);
-            mbar_init(&sm.d1_empty[b], kEpiWarps);
-            mbar_init(&sm.h_full[b], kEpiWarps);
-            mbar_init(&sm.h_empty[b], 1);
+        for (int q = 0; q < kW1Stages; ++q) { mbar_init(&sm.w1_full[q], 1); mbar_init(&sm.w1_empty[q], 1); }
+        for (int q = 0; q < kW2Stages; ++q) { mbar_init(&sm.w2_full[q], 1); mbar_init(&sm.w2_empty[q], 1); }
+        for (int q = 0; q < 2; ++q) {
+            mbar_init(&sm.a_full[q], 1);
+            mbar_init(&sm.a_empty[q], 1);
+            mbar_init(&sm.h_full[q], kEpiWarps);
+            mbar_init(&sm.h_empty[q], 1);
+        }
+        for (int q = 0; q < kD1Bufs; ++q) {
+            mbar_init(&sm.d1_full[q], 1);
+            mbar_init(&sm.d1_empty[q], kEpiWarps);
         }
         mbar_init(&sm.d2_full, 1);
         mbar_init(&sm.d2_empty, kEpiWarps);
@@ -174,151 +216,190 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     const uint32_t tmem = sm.tmem_base;
     const int n_my_tiles = (p.n_tiles > static_cast<int>(blockIdx.x)) ? (p.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
     const int NC = p.n_chunks;
+    const int n_my_chunks = n_my_tiles * NC;
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- weight producer
+        // ---------------------------------------------------------------- weight producers (lane 0: W1, lane 1: W2)
+        // The sum over hidden chunks may be taken in any order; each CTA starts at its own chunk so that the SMs do
+        // not all ask the same L2 lines for the same chunk at the same moment.
         if (lane == 0) {
-            int g = 0;      // running chunk count across tiles
-            for (int it = 0; it < n_my_tiles && !*abort_flag; ++it) {
-                for (int c = 0; c < NC; ++c, ++g) {
-                    const int s = g % kWStages;
-                    if (g >= kWStages && !mbar_wait(&sm.w_empty[s], static_cast<uint32_t>(g / kWStages - 1) & 1u, abort_flag)) break;
-                    mbar_expect_tx(&sm.w_full[s], kChunkBytes);
-                    bulk_load(sm.w[s], p.packed + static_cast<size_t>(c) * kChunkBytes, kChunkBytes, &sm.w_full[s]);
-                }
+            Ring<kW1Stages> r;
+            int cc = static_cast<int>(blockIdx.x) % NC;
+            for (int g = 0; g < n_my_chunks; ++g) {
+                if (r.wrapped && !mbar_wait(&sm.w1_empty[r.slot], r.phase ^ 1u, abort_flag)) break;
+                mbar_expect_tx(&sm.w1_full[r.slot], kTileBytes);
+                bulk_load(sm.w1[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes, kTileBytes, &sm.w1_full[r.slot]);
+                r.advance();
+                if (++cc == NC) cc = 0;
+            }
+        } else if (lane == 1) {
+            Ring<kW2Stages> r;
+            int cc = static_cast<int>(blockIdx.x) % NC;
+            for (int g = 0; g < n_my_chunks; ++g) {
+                if (r.wrapped && !mbar_wait(&sm.w2_empty[r.slot], r.phase ^ 1u, abort_flag)) break;
+                mbar_expect_tx(&sm.w2_full[r.slot], kTileBytes);
+                bulk_load(sm.w2[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes + kTileBytes, kTileBytes, &sm.w2_full[r.slot]);
+                r.advance();
+                if (++cc == NC) cc = 0;
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
+            // One thread issues every MMA, so its instruction stream is kept short: descriptors are a base word plus a
+            // constant, ring positions and phases are carried incrementally.
             constexpr uint32_t idesc1 = umma_idesc(kTok, kHc), idesc2 = umma_idesc(kTok, kCh);
-            const uint64_t a_desc = umma_desc(smem_u32(sm.a));
-            int g = 0;
+            constexpr uint32_t kTileUnits = kTileBytes >> 4;
+            const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]), w2_lo = desc_lo(sm.w2[0]), h_lo = desc_lo(sm.h[0][0]);
             bool ok = true;
-            // GEMM1 of chunk c of the current tile (global chunk index gc): D1[gc % 2] = A * W1_c
-            auto gemm1 = [&](int gc) -> bool {
-                const int s = gc % kWStages, b = gc & 1;
-                if (!mbar_wait(&sm.w_full[s], static_cast<uint32_t>(gc / kWStages) & 1u, abort_flag)) return false;
-                if (gc >= 2 && !mbar_wait(&sm.d1_empty[b], static_cast<uint32_t>(gc / 2 - 1) & 1u, abort_flag)) return false;
+            Ring<kW1Stages> rw1;      // weights of the next GEMM1
+            Ring<kD1Bufs> rd1;        // accumulator of the next GEMM1
+            Ring<kW2Stages> rw2;      // weights of the next GEMM2
+            Ring<2> rh;               // H buffer of the next GEMM2
+            uint32_t a_cur = a_lo;
+            auto gemm1 = [&]() -> bool {       // D1[rd1] = A * W1[rw1]
+                if (!mbar_wait(&sm.w1_full[rw1.slot], rw1.phase, abort_flag)) return false;
+                if (rd1.wrapped && !mbar_wait(&sm.d1_empty[rd1.slot], rd1.phase ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t b_desc = umma_desc(smem_u32(sm.w[s]));
+                const uint32_t b_lo = w1_lo + static_cast<uint32_t>(rw1.slot) * kTileUnits;
+                const uint32_t d = tmem + static_cast<uint32_t>(rd1.slot) * kHc;
 #pragma unroll
                 for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
-                    umma_bf16(tmem + static_cast<uint32_t>(b) * kHc, a_desc + 2u * k, b_desc + 2u * k, idesc1, k > 0 ? 1u : 0u);
-                umma_commit(&sm.d1_full[b]);
+                    umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
+                umma_commit(&sm.d1_full[rd1.slot]);
+                umma_commit(&sm.w1_empty[rw1.slot]);
+                rw1.advance();
+                rd1.advance();
                 return true;
             };
             for (int it = 0; it < n_my_tiles && ok; ++it) {
-                ok = mbar_wait(&sm.a_full, static_cast<uint32_t>(it) & 1u, abort_flag);
-                if (ok) ok = gemm1(g);
+                const int ab = it & 1;
+                ok = mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag);
+                a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
+                int issued1 = 0;                 // GEMM1s of this tile issued so far
+                while (ok && issued1 < NC && issued1 < 2) {
+                    ok = gemm1();
+                    if (++issued1 == NC) umma_commit(&sm.a_empty[ab]);   // every GEMM1 of this tile has been issued
+                }
                 for (int c = 0; c < NC && ok; ++c) {
-                    const int gc = g + c;
-                    if (c + 1 < NC) {
-                        ok = gemm1(gc + 1);
+                    if (issued1 < NC) {
+                        ok = gemm1();
                         if (!ok) break;
-                    } else {
-                        umma_commit(&sm.a_empty);          // every GEMM1 of this tile has been issued
+                        if (++issued1 == NC) umma_commit(&sm.a_empty[ab]);
                     }
-                    const int s = gc % kWStages, b = gc & 1;
-                    ok = mbar_wait(&sm.h_full[b], static_cast<uint32_t>(gc / 2) & 1u, abort_flag);
+                    ok = mbar_wait(&sm.h_full[rh.slot], rh.phase, abort_flag);
+                    if (ok) ok = mbar_wait(&sm.w2_full[rw2.slot], rw2.phase, abort_flag);
                     if (ok && c == 0 && it > 0) ok = mbar_wait(&sm.d2_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
+                    const uint32_t ha_lo = h_lo + static_cast<uint32_t>(rh.slot) * (2u * kTileUnits);
+                    const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(rw2.slot) * kTileUnits;
 #pragma unroll
-                    for (int k = 0; k < kHc / 16; ++k) {
-                        const uint64_t ha = umma_desc(smem_u32(sm.h[b][k / 4])) + 2u * (k % 4);
-                        const uint64_t wb = umma_desc(smem_u32(sm.w[s] + kHc * 128 + (k / 4) * (kCh * 128))) + 2u * (k % 4);
-                        umma_bf16(tmem + kD2Col, ha, wb, idesc2, (c > 0 || k > 0) ? 1u : 0u);
-                    }
-                    umma_commit(&sm.h_empty[b]);
-                    umma_commit(&sm.w_empty[s]);
+                    for (int k = 0; k < kHc / 16; ++k)
+                        umma_bf16(tmem + kD2Col, desc64(ha_lo + (k / 4) * kTileUnits + 2u * (k % 4)),
+                                  desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&sm.h_empty[rh.slot]);
+                    umma_commit(&sm.w2_empty[rw2.slot]);
                     if (c == NC - 1) umma_commit(&sm.d2_full);
+                    rh.advance();
+                    rw2.advance();
                 }
-                g += NC;
             }
         }
-    } else {
-        // ---------------------------------------------------------------- epilogue warps
-        const int ew = warp - 2;                  // 0..7
-        const uint32_t quarter = static_cast<uint32_t>(warp & 3);   // TMEM lanes this warp may touch: 32*quarter .. +31
-        const uint32_t half = static_cast<uint32_t>(ew >> 2);       // which 64 of the chunk's 128 columns
-        const uint32_t row = quarter * 32u + static_cast<uint32_t>(lane);       // token row of this thread in the tile
-        const uint32_t lane_addr = (quarter * 32u) << 16;
+    } else if (warp == kLoaderWarp) {
+        // ---------------------------------------------------------------- latent tile -> bf16, K-major swizzled
+        // The warp covers 2 rows per step (16 lanes x 16 B per row); 8 steps are in flight at a time.
         bool ok = true;
-        int g = 0;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
-            // ---- latent tile -> bf16, K-major swizzled.  A warp covers 2 rows per pass (16 lanes x 16 B per row).
-            if (it > 0) ok = mbar_wait(&sm.a_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;      // keep every verdict warp-uniform: the TMEM loads are warp-wide
+            const int ab = it & 1;
+            if (it >= 2) ok = mbar_wait(&sm.a_empty[ab], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
             if (!ok) break;
-            for (int pass = 0; pass < kTok / (2 * kEpiWarps); ++pass) {
-                const uint32_t r = static_cast<uint32_t>(pass * 2 * kEpiWarps + ew * 2 + (lane >> 4));
-                const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row
-                const int64_t q = tok0 + r;
-                float4 zv = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (q < p.n_tokens) {
-                    const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
-                    zv = __ldcs(reinterpret_cast<const float4*>(p.latents + tree * p.tree_stride + p.row_offset + rr * kCh) + c4);
+            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
+            const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row
+            unsigned char* atile = sm.a[ab];
+            for (int r0 = 0; r0 < kTok; r0 += 16) {
+                float4 zv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int64_t q = tok0 + r0 + 2 * u + (lane >> 4);
+                    zv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < p.n_tokens) {
+                        const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
+                        zv[u] = __ldcs(reinterpret_cast<const float4*>(p.latents + tree * p.tree_stride + p.row_offset + rr * kCh) + c4);
+                    }
                 }
-                uint2 packed2;
-                packed2.x = pack_bf16(zv.x, zv.y);
-                packed2.y = pack_bf16(zv.z, zv.w);
-                *reinterpret_cast<uint2*>(sm.a + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t r = static_cast<uint32_t>(r0 + 2 * u + (lane >> 4));
+                    uint2 packed2;
+                    packed2.x = pack_bf16(zv[u].x, zv[u].y);
+                    packed2.y = pack_bf16(zv[u].z, zv[u].w);
+                    *reinterpret_cast<uint2*>(atile + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
+                }
             }
             proxy_fence();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.a_full);
-
+            if (lane == 0) mbar_arrive(&sm.a_full[ab]);
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int ew = warp - 2;                  // 0..15
+        const uint32_t quarter = static_cast<uint32_t>(warp & 3);   // TMEM lanes this warp may touch: 32*quarter .. +31
+        const uint32_t sub = static_cast<uint32_t>(ew >> 2);        // which 32 of the chunk's 128 columns
+        const uint32_t row = quarter * 32u + static_cast<uint32_t>(lane);       // token row of this thread in the tile
+        const uint32_t lane_addr = (quarter * 32u) << 16;
+        bool ok = true;
+        Ring<kD1Bufs> rd1;
+        Ring<2> rh;
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
             for (int c = 0; c < NC && ok; ++c) {
-                const int gc = g + c, b = gc & 1;
-                ok = mbar_wait(&sm.d1_full[b], static_cast<uint32_t>(gc / 2) & 1u, abort_flag);
-                if (ok && gc >= 2) ok = mbar_wait(&sm.h_empty[b], static_cast<uint32_t>(gc / 2 - 1) & 1u, abort_flag);
-                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                ok = mbar_wait(&sm.d1_full[rd1.slot], rd1.phase, abort_flag);
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;      // keep every verdict warp-uniform: the TMEM loads are warp-wide
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll
-                for (int grp = 0; grp < 2; ++grp) {          // 2 x 32 columns of this warp's 64
-                    uint32_t acc[32];
-                    const uint32_t col = static_cast<uint32_t>(b) * kHc + half * 64u + static_cast<uint32_t>(grp) * 32u;
-                    tmem_ld32(tmem + lane_addr + col, acc);
-                    tmem_ld_wait();
-                    unsigned char* htile = sm.h[b][half];     // hidden columns half*64 .. +63 are K half `half` of GEMM2
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {             // 8 columns -> one 16-byte piece
-                        uint4 piece;
-                        piece.x = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 0])), gelu_fast(__uint_as_float(acc[8 * j + 1])));
-                        piece.y = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 2])), gelu_fast(__uint_as_float(acc[8 * j + 3])));
-                        piece.z = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 4])), gelu_fast(__uint_as_float(acc[8 * j + 5])));
-                        piece.w = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 6])), gelu_fast(__uint_as_float(acc[8 * j + 7])));
-                        *reinterpret_cast<uint4*>(htile + sw128(row, static_cast<uint32_t>(grp * 4 + j))) = piece;
-                    }
-                }
+                uint32_t acc[32];
+                tmem_ld32(tmem + lane_addr + static_cast<uint32_t>(rd1.slot) * kHc + sub * 32u, acc);
+                tmem_ld_wait();
                 tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.d1_empty[rd1.slot]);      // D1 is in registers: a later GEMM1 may overwrite it
+                rd1.advance();
+                if (rh.wrapped) ok = mbar_wait(&sm.h_empty[rh.slot], rh.phase ^ 1u, abort_flag);      // GEMM2 of chunk c - 2 has read this H buffer
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                if (!ok) break;
+                unsigned char* htile = sm.h[rh.slot][sub >> 1];    // hidden columns 0..63 / 64..127 are the two K halves of GEMM2
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {                      // 8 columns -> one 16-byte piece
+                    uint4 piece;
+                    piece.x = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 0])), gelu_fast(__uint_as_float(acc[8 * j + 1])));
+                    piece.y = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 2])), gelu_fast(__uint_as_float(acc[8 * j + 3])));
+                    piece.z = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 4])), gelu_fast(__uint_as_float(acc[8 * j + 5])));
+                    piece.w = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 6])), gelu_fast(__uint_as_float(acc[8 * j + 7])));
+                    *reinterpret_cast<uint4*>(htile + sw128(row, (sub & 1u) * 4u + static_cast<uint32_t>(j))) = piece;
+                }
                 proxy_fence();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&sm.d1_empty[b]);
-                    mbar_arrive(&sm.h_full[b]);
-                }
+                if (lane == 0) mbar_arrive(&sm.h_full[rh.slot]);
+                rh.advance();
             }
             if (!ok) break;
-            g += NC;
-            // ---- output tile: D2 -> v (this warp's 32 of the 64 channels)
+            // ---- output tile: D2 -> v (this warp's 16 of the 64 channels)
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.d2_full, static_cast<uint32_t>(it) & 1u, abort_flag) ? 1 : 0) != 0;
             if (!ok) break;
             tc_fence_after();
-            uint32_t out[32];
-            tmem_ld32(tmem + lane_addr + kD2Col + half * 32u, out);
+            uint32_t out[16];
+            tmem_ld16(tmem + lane_addr + kD2Col + sub * 16u, out);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.d2_empty);
             const int64_t q = tok0 + row;
             if (q < p.n_tokens) {
-                float4* dst = reinterpret_cast<float4*>(p.v_out + q * kCh + half * 32u);
+                float4* dst = reinterpret_cast<float4*>(p.v_out + q * kCh + sub * 16u);
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < 4; ++j)
                     dst[j] = make_float4(__uint_as_float(out[4 * j]), __uint_as_float(out[4 * j + 1]), __uint_as_float(out[4 * j + 2]),
                                          __uint_as_float(out[4 * j + 3]));
             }
