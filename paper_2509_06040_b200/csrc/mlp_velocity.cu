@@ -8,10 +8,11 @@
 //     GELU     : H_c = bf16(GELU(D1))   TMEM -> registers -> shared memory (the hidden activation never leaves the SM)
 //     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, accumulator in TMEM)
 // Warp roles:
-//     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 4-stage ring of W1 chunks,
-//                  lane 1 a 3-stage ring of W2 chunks (W1_c is needed two chunks earlier than W2_c);
-//     warp 1       owns tensor memory and issues every MMA from one thread; GEMM1 runs two chunks ahead (D1 is
-//                  triple-buffered), GEMM2(c) overlaps the epilogue of chunk c + 1 (H is double-buffered);
+//     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 3-stage ring of W1 chunks,
+//                  lane 1 a 2-stage ring of W2 chunks;
+//     warp 1       owns tensor memory; its lane 0 issues GEMM1, which runs up to three chunks ahead (D1 is
+//                  triple-buffered);
+//     warp 19      lane 0 issues GEMM2; GEMM2(c) overlaps the epilogue of chunk c + 1 (H is double-buffered);
 //     warps 2..17  GELU epilogue, four warps per TMEM lane quarter with 32 columns each, and the output tile;
 //     warp 18      converts the NEXT tile's latents to bf16 into the second A buffer while the current tile computes.
 // Operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors address; the
@@ -28,11 +29,12 @@ namespace {
 constexpr int kTok = 128;                 // tokens per tile = MMA M
 constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
 constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
-constexpr int kW1Stages = 4;
-constexpr int kW2Stages = 3;
+constexpr int kW1Stages = 3;               // = kD1Bufs: W1 slot q is free again when GEMM1 into D1[q] has completed
+constexpr int kW2Stages = 2;               // = H buffers: W2 slot q is free again when the GEMM2 reading H[q] has completed
 constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 32 columns of a chunk each
 constexpr int kLoaderWarp = 2 + kEpiWarps;
-constexpr int kMlpThreads = (3 + kEpiWarps) * 32;
+constexpr int kGemm2Warp = 3 + kEpiWarps;
+constexpr int kMlpThreads = (4 + kEpiWarps) * 32;
 constexpr uint32_t kTileBytes = kTok * 128;              // one [128 rows][128 B] operand tile = 16 KiB
 constexpr uint32_t kChunkBytes = 2 * kTileBytes;         // packed weights of a chunk: W1_c (16 KiB) then W2_c (16 KiB)
 constexpr int kD1Bufs = 3;                // GEMM1 runs two chunks ahead of the epilogue
@@ -45,7 +47,7 @@ struct MlpSmem {
     alignas(1024) unsigned char w2[kW2Stages][kTileBytes];  // W2_c as two [64 n = channel][128 B = 64 hidden] tiles
     alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
     alignas(1024) unsigned char h[2][2][kTileBytes];        // [buffer][k half][128 tok][128 B]
-    unsigned long long w1_full[kW1Stages], w1_empty[kW1Stages], w2_full[kW2Stages], w2_empty[kW2Stages];
+    unsigned long long w1_full[kW1Stages], w2_full[kW2Stages];
     unsigned long long a_full[2], a_empty[2], d1_full[kD1Bufs], d1_empty[kD1Bufs], h_full[2], h_empty[2], d2_full, d2_empty;
     uint32_t tmem_base;
     int abort_flag;
@@ -189,8 +191,8 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     volatile int* abort_flag = &sm.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int q = 0; q < kW1Stages; ++q) { mbar_init(&sm.w1_full[q], 1); mbar_init(&sm.w1_empty[q], 1); }
-        for (int q = 0; q < kW2Stages; ++q) { mbar_init(&sm.w2_full[q], 1); mbar_init(&sm.w2_empty[q], 1); }
+        for (int q = 0; q < kW1Stages; ++q) mbar_init(&sm.w1_full[q], 1);
+        for (int q = 0; q < kW2Stages; ++q) mbar_init(&sm.w2_full[q], 1);
         for (int q = 0; q < 2; ++q) {
             mbar_init(&sm.a_full[q], 1);
             mbar_init(&sm.a_empty[q], 1);
@@ -226,7 +228,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             Ring<kW1Stages> r;
             int cc = static_cast<int>(blockIdx.x) % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
-                if (r.wrapped && !mbar_wait(&sm.w1_empty[r.slot], r.phase ^ 1u, abort_flag)) break;
+                if (r.wrapped && !mbar_wait(&sm.d1_full[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM1 that read this slot is done
                 mbar_expect_tx(&sm.w1_full[r.slot], kTileBytes);
                 bulk_load(sm.w1[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes, kTileBytes, &sm.w1_full[r.slot]);
                 r.advance();
@@ -236,7 +238,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             Ring<kW2Stages> r;
             int cc = static_cast<int>(blockIdx.x) % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
-                if (r.wrapped && !mbar_wait(&sm.w2_empty[r.slot], r.phase ^ 1u, abort_flag)) break;
+                if (r.wrapped && !mbar_wait(&sm.h_empty[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM2 that read this slot is done
                 mbar_expect_tx(&sm.w2_full[r.slot], kTileBytes);
                 bulk_load(sm.w2[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes + kTileBytes, kTileBytes, &sm.w2_full[r.slot]);
                 r.advance();
@@ -244,65 +246,60 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             }
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
+        // ---------------------------------------------------------------- GEMM1 issuer
+        // Two threads issue MMAs, one per GEMM, so that a GEMM1 held back by the tensor pipe never delays the GEMM2 the
+        // epilogue is waiting for (and vice versa); completion tracking (tcgen05.commit) is per issuing thread.
         if (lane == 0) {
-            // One thread issues every MMA, so its instruction stream is kept short: descriptors are a base word plus a
-            // constant, ring positions and phases are carried incrementally.
-            constexpr uint32_t idesc1 = umma_idesc(kTok, kHc), idesc2 = umma_idesc(kTok, kCh);
+            constexpr uint32_t idesc1 = umma_idesc(kTok, kHc);
             constexpr uint32_t kTileUnits = kTileBytes >> 4;
-            const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]), w2_lo = desc_lo(sm.w2[0]), h_lo = desc_lo(sm.h[0][0]);
+            static_assert(kW1Stages == kD1Bufs, "the W1 ring and the D1 ring advance together");
+            const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]);
             bool ok = true;
-            Ring<kW1Stages> rw1;      // weights of the next GEMM1
-            Ring<kD1Bufs> rd1;        // accumulator of the next GEMM1
-            Ring<kW2Stages> rw2;      // weights of the next GEMM2
-            Ring<2> rh;               // H buffer of the next GEMM2
-            uint32_t a_cur = a_lo;
-            auto gemm1 = [&]() -> bool {       // D1[rd1] = A * W1[rw1]
-                if (!mbar_wait(&sm.w1_full[rw1.slot], rw1.phase, abort_flag)) return false;
-                if (rd1.wrapped && !mbar_wait(&sm.d1_empty[rd1.slot], rd1.phase ^ 1u, abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t b_lo = w1_lo + static_cast<uint32_t>(rw1.slot) * kTileUnits;
-                const uint32_t d = tmem + static_cast<uint32_t>(rd1.slot) * kHc;
-#pragma unroll
-                for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
-                    umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
-                umma_commit(&sm.d1_full[rd1.slot]);
-                umma_commit(&sm.w1_empty[rw1.slot]);
-                rw1.advance();
-                rd1.advance();
-                return true;
-            };
+            Ring<kD1Bufs> r;          // weights and accumulator of the next GEMM1
             for (int it = 0; it < n_my_tiles && ok; ++it) {
                 const int ab = it & 1;
                 ok = mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag);
-                a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
-                int issued1 = 0;                 // GEMM1s of this tile issued so far
-                while (ok && issued1 < NC && issued1 < 2) {
-                    ok = gemm1();
-                    if (++issued1 == NC) umma_commit(&sm.a_empty[ab]);   // every GEMM1 of this tile has been issued
+                const uint32_t a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
+                for (int c = 0; c < NC && ok; ++c) {       // D1[r] = A * W1[r]
+                    ok = mbar_wait(&sm.w1_full[r.slot], r.phase, abort_flag);
+                    if (ok && r.wrapped) ok = mbar_wait(&sm.d1_empty[r.slot], r.phase ^ 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t b_lo = w1_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
+                    const uint32_t d = tmem + static_cast<uint32_t>(r.slot) * kHc;
+#pragma unroll
+                    for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
+                        umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
+                    umma_commit(&sm.d1_full[r.slot]);
+                    r.advance();
                 }
-                for (int c = 0; c < NC && ok; ++c) {
-                    if (issued1 < NC) {
-                        ok = gemm1();
-                        if (!ok) break;
-                        if (++issued1 == NC) umma_commit(&sm.a_empty[ab]);
-                    }
-                    ok = mbar_wait(&sm.h_full[rh.slot], rh.phase, abort_flag);
-                    if (ok) ok = mbar_wait(&sm.w2_full[rw2.slot], rw2.phase, abort_flag);
+                if (ok) umma_commit(&sm.a_empty[ab]);       // every GEMM1 of this tile has been issued
+            }
+        }
+    } else if (warp == kGemm2Warp) {
+        // ---------------------------------------------------------------- GEMM2 issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc2 = umma_idesc(kTok, kCh);
+            constexpr uint32_t kTileUnits = kTileBytes >> 4;
+            const uint32_t w2_lo = desc_lo(sm.w2[0]), h_lo = desc_lo(sm.h[0][0]);
+            bool ok = true;
+            Ring<2> r;                // H buffer and weights of the next GEMM2
+            for (int it = 0; it < n_my_tiles && ok; ++it) {
+                for (int c = 0; c < NC && ok; ++c) {       // D2 += H[r] * W2[r]
+                    ok = mbar_wait(&sm.w2_full[r.slot], r.phase, abort_flag);
+                    if (ok) ok = mbar_wait(&sm.h_full[r.slot], r.phase, abort_flag);
                     if (ok && c == 0 && it > 0) ok = mbar_wait(&sm.d2_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t ha_lo = h_lo + static_cast<uint32_t>(rh.slot) * (2u * kTileUnits);
-                    const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(rw2.slot) * kTileUnits;
+                    const uint32_t ha_lo = h_lo + static_cast<uint32_t>(r.slot) * (2u * kTileUnits);
+                    const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
 #pragma unroll
                     for (int k = 0; k < kHc / 16; ++k)
                         umma_bf16(tmem + kD2Col, desc64(ha_lo + (k / 4) * kTileUnits + 2u * (k % 4)),
                                   desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&sm.h_empty[rh.slot]);
-                    umma_commit(&sm.w2_empty[rw2.slot]);
+                    umma_commit(&sm.h_empty[r.slot]);
                     if (c == NC - 1) umma_commit(&sm.d2_full);
-                    rh.advance();
-                    rw2.advance();
+                    r.advance();
                 }
             }
         }
