@@ -37,10 +37,16 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload; reported only while the kernel source still has the
-# hash the capture was taken with.  Filled in from profiles/.
-NCU_TRAFFIC = {}
+# DRAM traffic of the dominant kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum), see
+# profiles/.  Each entry is the captured launch's bytes and the units (elements / tokens) it processed; the figure
+# reported per launch is bytes-per-unit times the units of an average launch of the timed workload (traffic grows in
+# proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
+NCU_TRAFFIC = {
+    "step_kernel": {"workload": "video", "bytes": 75.599104e6 + 12.592896e6, "units": 8 * 2096640,
+                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "d6ef704e319c"},
+    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.249216e6 + 212.080384e6, "units": 1036800,
+                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "ca53c8c3093c"},
+}
 
 
 def load_peaks():
@@ -75,6 +81,23 @@ def step_bytes_per_launch(w, n_trees):
         out.append(b)
         width *= fan
     return out
+
+
+def step_children(w):
+    """Children written by each tree_step launch of the batch (n_trees * W_{i+1})."""
+    out, width = [], 1
+    for i in range(w.T):
+        width *= (w.K if i in w.splits else 1)
+        out.append(w.n_trees * width)
+    return out
+
+
+def ncu_traffic(kernel, units_per_launch):
+    """DRAM bytes of an average launch, scaled from the committed ncu capture; None once the kernel has changed."""
+    tr = NCU_TRAFFIC[kernel]
+    if tr["source_hash"] != kernel_source_hash(tr["sources"]):
+        return None
+    return tr["bytes"] / tr["units"] * units_per_launch
 
 
 def mlp_flops_per_launch(w, n_trees):
@@ -353,9 +376,7 @@ def run_ours(args, w):
                      "widest_launch": {"step": widest, "bytes": float(sb[widest]), "ms": float(t_step[widest]),
                                        "gbs": float(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
                      "traffic": None}
-        tr = NCU_TRAFFIC.get(w.name)
-        if tr and tr.get("source_hash") == kernel_source_hash():
-            roof_step["traffic"] = tr["bytes_per_launch"]
+        roof_step["traffic"] = ncu_traffic("step_kernel", float(sum(n_trees_w * w.D for n_trees_w in step_children(w))) / w.T)
         breakdown = {"step_ms": float(t_step.sum()), "mlp_ms": float(t_mlp.sum()), "other_ms": float(t_other)}
         if w.velocity == "mlp" and t_mlp.sum() > t_step.sum():
             fl = np.array(mlp_flops_per_launch(w, w.n_trees), dtype=np.float64)
@@ -363,7 +384,8 @@ def run_ours(args, w):
             peak_tf = float(peaks["bf16_tflops"])
             roof = {"bound": "tensor", "kernel": "mlp_velocity_kernel", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": tf / peak_tf, "peak_source": peaks["_source"], "launches_per_pass": w.T,
-                    "flops_per_pass": float(fl.sum()), "ms_per_pass": float(t_mlp.sum()), "traffic": None}
+                    "flops_per_pass": float(fl.sum()), "ms_per_pass": float(t_mlp.sum()),
+                    "traffic": ncu_traffic("mlp_velocity_kernel", float(w.n_trees * w.model_evals * w.tokens) / w.T)}
         else:
             roof = roof_step
 

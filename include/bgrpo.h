@@ -131,8 +131,11 @@ bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* tree, const float* mu_dev, f
  * the rectified-flow SDE, mu_theta = z - h v - (sigma^2 h / (2 t)) (z + (1-t) v), evaluated once per parent.
  * v_dev: device [n_trees][W_i][D] velocities of the current frontier (e.g. from bgrpo_velocity_mlp), or NULL for the
  * bound linear velocity.  One fused kernel appends the children's node-table rows, writes their latents and the
- * per-element-mean Gaussian log-prob of each new edge,
+ * partial sums of the per-element-mean Gaussian log-prob of each new edge,
  *   logp = -(1/D) sum_e (z'_e - mu_e)^2 / (2 g_i^2) - ln g_i - 0.5 ln(2 pi)      (multiply by D for the joint density).
+ * The sums are completed, in a fixed order, by the next call for this tree that is enqueued on the stream (the next
+ * tree_step's kernel does it in its prologue) and at the latest by the step that completes the tree, which enqueues a
+ * small flush kernel: buffers.logp of a level is final once one of those has run.  Use one stream per tree handle.
  * Errors: STATE (already at depth T; NULL v_dev without a bound velocity), CAPACITY (children exceed nodes_cap), CUDA. */
 bgrpo_status bgrpo_tree_step(bgrpo_tree* tree, int32_t split_flag, const float* v_dev, void* stream);
 
