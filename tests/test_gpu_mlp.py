@@ -61,6 +61,7 @@ def test_mlp_stage_matches_oracle_at_every_depth(B, tokens, hidden, n_trees, K, 
         worst = max(worst, err / rms)
         B.tree_step(s.tree, 1 if i in w.splits else 0, torch.from_numpy(ref).cuda())
     torch.cuda.synchronize()
+    print("worst |d| / rms(v) over the depths:", worst)
     assert worst < 2e-2
     # the teacher-forced steps reproduce the oracle's latents
     for t in range(n_trees):
