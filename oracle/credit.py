@@ -119,9 +119,12 @@ def depth_keep(topo: Topology, pruned_steps: Iterable[int]) -> np.ndarray:
 
 
 def gradient_mask(topo: Topology, rbar: np.ndarray, width_mode: int, k: int,
-                  pruned_steps: Iterable[int] = (), ignore_last_step: bool = False) -> np.ndarray:
-    """mask[n] = 1 iff the node-step (edge) into n receives gradients."""
+                  pruned_steps: Iterable[int] = (), ignore_last_step: bool = False, sde_steps=None) -> np.ndarray:
+    """mask[n] = 1 iff the node-step (edge) into n receives gradients.  With a hybrid ODE-SDE
+    schedule (sde_steps given) the deterministic ODE steps have no transition density and are masked."""
     m = width_keep(topo, rbar, width_mode, k) & depth_keep(topo, pruned_steps)
+    if sde_steps is not None:
+        m &= depth_keep(topo, [i for i in range(topo.T) if i not in set(int(x) for x in sde_steps)])
     m[0] = 0
     if ignore_last_step:   # "Ignore last step: Yes" (hyper-parameter table)
         m[list(topo.level(topo.T))] = 0
@@ -134,3 +137,28 @@ def depth_window(iteration: int, start: int, size: int = 4, every: int = 30, sto
     if stop is not None:
         first = min(first, stop - size)
     return [first + j for j in range(size)]
+
+
+def grpo_objective(topo: Topology, logp_new: np.ndarray, logp_old: np.ndarray, adv: np.ndarray, mask: np.ndarray,
+                   clip_eps: float, logp_scale: float = 1.0):
+    """Forward value of the clipped GRPO objective over the tree's edges (Eq. 5):
+        J = 1/|E| sum_e min(rho_e A(e), clip(rho_e, 1 - eps, 1 + eps) A(e)),   rho_e = pi_new(e) / pi_old(e),
+    with E the edges that receive gradients (mask) and rho_e = exp(logp_scale (logp_new - logp_old)).
+    Returns (J, per-edge terms with 0 on unmasked nodes).  An empty edge set gives J = 0."""
+    terms = np.zeros(topo.nodes, dtype=np.float64)
+    n = 0
+    for e in range(1, topo.nodes):
+        if not mask[e]:
+            continue
+        rho = math.exp(logp_scale * (float(logp_new[e]) - float(logp_old[e])))
+        a = float(adv[e])
+        terms[e] = min(rho * a, min(max(rho, 1.0 - clip_eps), 1.0 + clip_eps) * a)
+        n += 1
+    return (float(terms.sum() / n) if n else 0.0), terms
+
+
+def mix_sde_steps(T: int, splits: Sequence[int], iteration: int, window: int = 4, every: int = 30, start: int = 0):
+    """Hybrid ODE-SDE schedule: every branching step plus a sliding window of `window` further steps (same
+    window rule as depth pruning: one step deeper every `every` iterations, kept inside 0..T-1)."""
+    first = min(start + iteration // every, max(T - window, 0))
+    return sorted(set(int(x) for x in splits) | set(range(first, min(first + window, T))))

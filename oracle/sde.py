@@ -92,7 +92,7 @@ VelocityFn = Callable[[np.ndarray, int, int], np.ndarray]
 
 def rollout(topo: Topology, n_elem: int, t_grid, sigma: float, s: float, seed: int,
             velocity_fn: VelocityFn, tree_id: int = 0, nodes_cap: Optional[int] = None,
-            elem_start: int = 0, return_means: bool = False):
+            elem_start: int = 0, return_means: bool = False, sde_steps=None):
     """Grow one tree (Algorithm 1, "Build rollout tree"): the root from the ROOT stream,
     then for i = 0..T-1 every node of depth i is advanced once, to K children at a split
     step and to one child otherwise.
@@ -100,6 +100,11 @@ def rollout(topo: Topology, n_elem: int, t_grid, sigma: float, s: float, seed: i
     n_elem elements starting at element index elem_start of each latent row are
     computed (the whole row by default); log-probs are only meaningful for whole rows.
     Global node id (the Philox counter word) = tree_id * nodes_cap + local index.
+
+    sde_steps: the hybrid ODE-SDE schedule of the ablation "Hybrid ODE-SDE" (all branching steps
+    stay SDE, a window picks further SDE steps, the remaining updates are ODE steps): an iterable
+    of the steps that are stochastic; None = all.  An ODE step uses sigma = 0 (drift -v, no noise,
+    log-prob 0); a split step must be an SDE step.
 
     Returns (latents float32 [nodes][n_elem], logp float64 [nodes]) and, on request,
     the float64 means of every non-root node.
@@ -112,10 +117,14 @@ def rollout(topo: Topology, n_elem: int, t_grid, sigma: float, s: float, seed: i
     logp = np.zeros(topo.nodes, dtype=np.float64)
     means = np.zeros((topo.nodes, n_elem), dtype=np.float64) if return_means else None
     lat[0] = root_latent(seed, base, n_elem, elem_start)
+    sde = None if sde_steps is None else set(int(x) for x in sde_steps)
+    sigma_all = sigma
     for i in range(topo.T):
         h = float(t[i] - t[i + 1])
-        g = noise_scale(sigma, h)
+        sigma = sigma_all if (sde is None or i in sde) else 0.0
         is_split = i in topo.splits
+        assert not (is_split and sigma == 0.0 and sigma_all != 0.0), "a split step must be an SDE step"
+        g = noise_scale(sigma, h)
         for p in topo.level(i):
             z = lat[p].astype(np.float64)
             v = np.asarray(velocity_fn(lat[p], i, p), dtype=np.float64)

@@ -194,3 +194,48 @@ def test_sliding_window_schedule():
     assert credit.depth_window(95, 9, stop=16) == [12, 13, 14, 15]
     assert credit.depth_window(3000, 9, stop=16) == [12, 13, 14, 15]
     assert credit.depth_window(61, 10, size=2, every=20) == [13, 14]
+
+
+def test_grpo_objective_equals_library_clipped_surrogate():
+    """Eq. 5 against the clipped surrogate composed from torch primitives, and its textbook cases."""
+    import torch
+    topo, r, logp_old = _random_case(6, 2, (0, 2, 4), seed=21)
+    rng = np.random.default_rng(3)
+    logp_new = logp_old + 0.3 * rng.standard_normal(topo.nodes)
+    rbar = credit.fuse_rewards(topo, r, logp_old, 1.0)
+    adv = credit.depth_advantages(topo, rbar, 1e-6)
+    mask = credit.gradient_mask(topo, rbar, credit.WIDTH_PER_SPLIT_TOPK, 1, [1, 4])
+    for eps, scale in ((0.2, 1.0), (1e-4, 1.0), (0.1, 3.0)):
+        J, terms = credit.grpo_objective(topo, logp_new, logp_old, adv, mask, eps, scale)
+        ratio = torch.exp(torch.tensor(scale * (logp_new - logp_old)))
+        A = torch.tensor(adv)
+        ref = torch.minimum(ratio * A, torch.clamp(ratio, 1 - eps, 1 + eps) * A)
+        sel = torch.tensor(mask.astype(bool))
+        sel[0] = False
+        assert math.isclose(J, float(ref[sel].mean()), rel_tol=1e-12, abs_tol=1e-15)
+        assert np.allclose(terms[mask.astype(bool)], ref[sel].numpy(), rtol=1e-12)
+        assert np.all(terms[~mask.astype(bool)] == 0)
+    # new policy == old policy: rho = 1, J = mean advantage over the edge set; over ALL edges the depth-wise
+    # standardisation makes every depth sum to zero, so J = 0
+    full = np.ones(topo.nodes, dtype=np.uint8)
+    J, _ = credit.grpo_objective(topo, logp_old, logp_old, adv, full, 0.2)
+    assert abs(J) < 1e-12
+    # the three regimes of the clip for one edge
+    one = tree.build_topology(1, 1, ())
+    for a, dl, eps, expect in ((2.0, 0.5, 0.2, 1.2 * 2.0), (-2.0, -0.5, 0.2, 0.8 * -2.0), (2.0, -0.5, 0.2, math.exp(-0.5) * 2.0),
+                               (-2.0, 0.5, 0.2, math.exp(0.5) * -2.0)):
+        J, _ = credit.grpo_objective(one, np.array([0.0, dl]), np.zeros(2), np.array([0.0, a]), np.array([0, 1]), eps)
+        assert math.isclose(J, expect, rel_tol=1e-12)
+    assert credit.grpo_objective(one, np.zeros(2), np.zeros(2), np.ones(2), np.zeros(2, dtype=np.uint8), 0.2)[0] == 0.0
+
+
+def test_mix_schedule():
+    """All branching steps stay SDE; a window of 4 adds further SDE steps and slides every 30 iterations."""
+    assert credit.mix_sde_steps(20, (0, 3, 6, 9), 0) == [0, 1, 2, 3, 6, 9]
+    assert credit.mix_sde_steps(20, (0, 3, 6, 9), 30 * 5) == [0, 3, 5, 6, 7, 8, 9]
+    assert credit.mix_sde_steps(20, (0, 3, 6, 9), 10 ** 6) == [0, 3, 6, 9, 16, 17, 18, 19]
+    topo = tree.build_topology(8, 2, (0, 3))
+    rbar = np.zeros(topo.nodes)
+    m = credit.gradient_mask(topo, rbar, credit.WIDTH_NONE, 0, (), False, sde_steps=[0, 3, 5])
+    for n in range(1, topo.nodes):
+        assert m[n] == int(topo.depth[n] - 1 in (0, 3, 5))

@@ -184,3 +184,43 @@ def test_element_slices_agree_with_whole_rows():
     full, _ = sde.rollout(topo, n, g, 0.3, 2.0, seed=1, velocity_fn=_vel(mu, g))
     part, _ = sde.rollout(topo, 64, g, 0.3, 2.0, seed=1, velocity_fn=_vel(mu[128:192], g), elem_start=128)
     assert np.array_equal(part, full[:, 128:192])
+
+
+def test_hybrid_ode_sde_schedule():
+    """ODE steps are deterministic (child = mean, log-prob 0), SDE steps unchanged, and a hybrid schedule still
+    carries N(0,1) onto N(mu, s0^2) in the limit (every step, ODE or SDE, preserves the marginals)."""
+    T, n = 6, 4096
+    g = _grid(T)
+    mu = np.zeros(n)
+    topo = tree.build_topology(T, 2, (0, 3))
+    sde_steps = [0, 3, 4]
+    lat, logp, means = sde.rollout(topo, n, g, 0.3, math.inf, seed=9, velocity_fn=_vel(mu, g), return_means=True, sde_steps=sde_steps)
+    full, logp_full = sde.rollout(topo, n, g, 0.3, math.inf, seed=9, velocity_fn=_vel(mu, g))
+    for c in range(1, topo.nodes):
+        i = int(topo.depth[c]) - 1
+        if i in sde_steps:
+            assert logp[c] != 0.0 and not np.array_equal(lat[c], means[c].astype(np.float32))
+        else:
+            assert logp[c] == 0.0 and np.array_equal(lat[c], means[c].astype(np.float32))
+    # the first step is SDE in both runs and draws the same noise
+    assert np.array_equal(lat[1], full[1]) and logp[1] == logp_full[1]
+    # all-ODE equals the sigma = 0 rollout
+    a, _ = sde.rollout(tree.build_topology(T, 2, ()), 64, g, 0.3, math.inf, seed=9, velocity_fn=_vel(mu[:64], g), sde_steps=[])
+    b, _ = sde.rollout(tree.build_topology(T, 2, ()), 64, g, 0.0, math.inf, seed=9, velocity_fn=_vel(mu[:64], g))
+    assert np.array_equal(a, b)
+    # marginal preservation with every other step stochastic
+    gaps = []
+    for TT in (256, 2048):
+        gg = _grid(TT)
+        P, V = 1.0, 0.0
+        for i in range(TT):
+            t, h = gg[i], gg[i] - gg[i + 1]
+            sig = 0.5 if i % 2 == 0 else 0.0
+            f = lambda z: sde.em_mean(np.array([z]), sde.linear_velocity(np.array([z]), t, np.array([0.0]), S0), t, h, sig)[0]
+            a_ = f(1.0) - f(0.0)
+            P *= a_
+            V = a_ * a_ * V + sde.noise_scale(sig, h) ** 2
+        gaps.append(abs(P * P + V - S0 ** 2))
+    assert gaps[1] < gaps[0] and gaps[1] < 5e-4
+    with pytest.raises(AssertionError):
+        sde.rollout(topo, 8, g, 0.3, math.inf, seed=9, velocity_fn=_vel(mu[:8], g), sde_steps=[3])   # split step 0 must be SDE
