@@ -181,6 +181,27 @@ bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* tree, const float* leaf_rewar
 bgrpo_status bgrpo_tree_prune(bgrpo_tree* tree, int32_t width_mode, int32_t k_or_b, const int32_t* pruned_steps_host,
                               int32_t n_pruned, int32_t ignore_last_step, void* stream);
 
+/* Clipped GRPO objective over the tree's edges, forward value (Eq. 5):
+ *   J = 1/|E| sum_e min(rho_e A(e), clip(rho_e, 1 - clip_eps, 1 + clip_eps) A(e)),  rho_e = exp(logp_scale (logp_new(e) - logp_old(e))),
+ * per tree, with E the node-steps whose buffers.mask is 1 and A = buffers.adv (so call it after tree_fuse_advantage and
+ * tree_prune).  logp_new_dev: device [n_trees][nodes_cap], e.g. from bgrpo_tree_logprob under the new policy's velocity;
+ * logp_old_dev: the behaviour policy's log-probs, NULL = buffers.logp; logp_scale: D turns per-element means into joint
+ * log-densities.  terms_out_dev: device [n_trees][nodes_cap] per-edge summands (0 where the mask is 0), may be NULL;
+ * J_out_dev: device [n_trees] float32 (0 for a tree with no masked edge).  STATE unless the tree is complete. */
+bgrpo_status bgrpo_tree_grpo_objective(bgrpo_tree* tree, const float* logp_new_dev, const float* logp_old_dev, float logp_scale,
+                                       float clip_eps, float* terms_out_dev, float* J_out_dev, void* stream);
+
+/* Hybrid ODE-SDE schedule (ablation "Hybrid ODE-SDE": all branching steps are preserved as SDE, a sliding window determines
+ * additional SDE steps, the remaining updates are ODE steps).  sde_flags_host: host array of T bytes, 1 = step i is
+ * stochastic, 0 = deterministic (sigma = 0 for that step: drift -v only, no noise drawn, log-prob written as 0, and
+ * tree_prune masks its node-steps); NULL restores "every step is SDE".  Host only; affects the steps taken afterwards.
+ * A later tree_step with split_flag != 0 on an ODE step returns INVALID_ARG (identical children carry no signal). */
+bgrpo_status bgrpo_tree_set_sde_steps(bgrpo_tree* tree, const uint8_t* sde_flags_host);
+/* The schedule itself: flags_out[i] = 1 for every split step and for the window steps
+ * min(start + iter/every, T - window) + 0..window-1.  Host only; flags_out holds T bytes. */
+bgrpo_status bgrpo_mix_sde_steps(int32_t T, const int32_t* split_steps, int32_t n_splits, int32_t iter, int32_t window,
+                                 int32_t every, int32_t start, uint8_t* flags_out);
+
 /* Sliding-window schedule of depth pruning (ablation "Pruning Strategies": window initialised at the last split point,
  * size 4, one step deeper every 30 iterations, until a stop depth): steps_out[j] = min(start + iter/every, stop-size) + j.
  * stop < 0 = no stop.  Host only; steps_out holds `size` entries. */

@@ -71,6 +71,9 @@ _SIGNATURES = {
     "bgrpo_leaf_reward_cos": (C.c_int, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_fuse_advantage": (C.c_int, [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_float, C.c_void_p]),
     "bgrpo_tree_prune": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, _i32p, C.c_int32, C.c_int32, C.c_void_p]),
+    "bgrpo_tree_grpo_objective": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "bgrpo_tree_set_sde_steps": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "bgrpo_mix_sde_steps": (C.c_int, [C.c_int32, _i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "bgrpo_depth_window": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _i32p, _i32p]),
     "bgrpo_tree_stats": (C.c_int, [C.c_void_p, _i32p, _i64p, _i64p, _i64p, _i64p]),
     "bgrpo_tree_levels": (C.c_int, [C.c_void_p, C.c_int32, _i32p, _i32p]),
@@ -202,6 +205,24 @@ def tree_prune(tree: Tree, width_mode: int, k_or_b: int, pruned_steps: Sequence[
     arr = (C.c_int32 * max(1, n))(*[int(x) for x in pruned_steps])
     _check(lib.bgrpo_tree_prune(tree.handle, width_mode, k_or_b, arr, n, int(bool(ignore_last_step)), _stream(stream)),
            "bgrpo_tree_prune")
+
+
+def tree_grpo_objective(tree: Tree, logp_new, logp_old=None, logp_scale=1.0, clip_eps=1e-4, terms_out=None, J_out=None,
+                        stream=None):
+    _check(lib.bgrpo_tree_grpo_objective(tree.handle, _ptr(logp_new), _ptr(logp_old), logp_scale, clip_eps, _ptr(terms_out),
+                                         _ptr(J_out), _stream(stream)), "bgrpo_tree_grpo_objective")
+
+
+def tree_set_sde_steps(tree: Tree, sde_flags: Optional[Sequence[int]]):
+    arr = None if sde_flags is None else np.ascontiguousarray(sde_flags, dtype=np.uint8)
+    _check(lib.bgrpo_tree_set_sde_steps(tree.handle, None if arr is None else arr.ctypes.data), "bgrpo_tree_set_sde_steps")
+
+
+def mix_sde_steps(T: int, split_steps: Sequence[int], iteration: int, window: int = 4, every: int = 30, start: int = 0):
+    arr = (C.c_int32 * max(1, len(split_steps)))(*[int(x) for x in split_steps])
+    out = np.zeros(T, dtype=np.uint8)
+    _check(lib.bgrpo_mix_sde_steps(T, arr, len(split_steps), iteration, window, every, start, out.ctypes.data), "bgrpo_mix_sde_steps")
+    return [i for i in range(T) if out[i]]
 
 
 def depth_window(iteration: int, start: int, size: int = 4, every: int = 30, stop: int = -1):

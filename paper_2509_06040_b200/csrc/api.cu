@@ -54,8 +54,8 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
 }
 
 void fill_coefficients(bgrpo_tree* t) {
-    const double sigma = t->desc.sigma;
     for (int i = 0; i < t->desc.T; ++i) {
+        const double sigma = ((t->ode_bits >> i) & 1ull) ? 0.0 : static_cast<double>(t->desc.sigma);   // ODE steps of the hybrid schedule
         const double ti = t->t_grid[i], h = static_cast<double>(t->t_grid[i]) - static_cast<double>(t->t_grid[i + 1]);
         const double c = sigma * sigma * h / (2.0 * ti);
         const double a = 1.0 - c, b = -(h + c * (1.0 - ti));
@@ -183,6 +183,7 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     }
     t->mu = nullptr;
     t->s0 = 0.0f;
+    t->ode_bits = 0;
     char* sc = static_cast<char*>(b->scratch);
     const size_t rows = static_cast<size_t>(desc->n_trees) * desc->nodes_cap;
     t->status = reinterpret_cast<int32_t*>(sc);
@@ -255,6 +256,8 @@ bgrpo_status bgrpo_tree_step(bgrpo_tree* t, int32_t split_flag, const float* v_d
     if (!v_dev && !t->mu) return fail(BGRPO_ERR_STATE, "no velocity: pass v_dev or bind a linear velocity");
     if (v_dev && !aligned(v_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "v misaligned");
     const int i = t->depth;
+    if (split_flag && ((t->ode_bits >> i) & 1ull) && t->desc.sigma > 0.0f)
+        return fail(BGRPO_ERR_INVALID_ARG, "a split step must be an SDE step of the hybrid schedule");
     const int fan = split_flag ? t->desc.K : 1;
     const int64_t W_out = static_cast<int64_t>(t->lv.width[i]) * fan;
     const int64_t off_out = t->lv.offset[i + 1];
@@ -380,7 +383,7 @@ bgrpo_status bgrpo_tree_prune(bgrpo_tree* t, int32_t width_mode, int32_t k_or_b,
     if (width_mode != BGRPO_WIDTH_NONE && k_or_b < 1) return fail(BGRPO_ERR_INVALID_ARG, "k_or_b must be >= 1");
     if (n_pruned < 0 || (n_pruned > 0 && !pruned_steps_host)) return fail(BGRPO_ERR_INVALID_ARG, "bad pruned_steps");
     PruneLaunch p;
-    p.pruned_bits = 0;
+    p.pruned_bits = t->ode_bits;      // deterministic steps have no transition density: never in the edge set
     for (int q = 0; q < n_pruned; ++q) {
         if (pruned_steps_host[q] < 0 || pruned_steps_host[q] >= t->desc.T) return fail(BGRPO_ERR_INVALID_ARG, "pruned step out of range");
         p.pruned_bits |= 1ull << pruned_steps_host[q];
@@ -402,6 +405,54 @@ bgrpo_status bgrpo_tree_prune(bgrpo_tree* t, int32_t width_mode, int32_t k_or_b,
     if (static_cast<size_t>(p.nodes) > 200 * 1024) return fail(BGRPO_ERR_UNSUPPORTED, "tree too large for one CTA's shared memory");
     cudaError_t e = launch_prune(p, as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "prune kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_grpo_objective(bgrpo_tree* t, const float* logp_new_dev, const float* logp_old_dev, float logp_scale,
+                                       float clip_eps, float* terms_out_dev, float* J_out_dev, void* stream) {
+    if (!t || !logp_new_dev || !J_out_dev) return fail(BGRPO_ERR_INVALID_ARG, "tree, logp_new or J_out is NULL");
+    if (!tree_complete(t)) return fail(BGRPO_ERR_STATE, "tree is not complete");
+    if (!std::isfinite(logp_scale) || !(clip_eps >= 0.0f) || !std::isfinite(clip_eps)) return fail(BGRPO_ERR_INVALID_ARG, "logp_scale must be finite and clip_eps >= 0");
+    ObjectiveLaunch p;
+    p.logp_new = logp_new_dev;
+    p.logp_old = logp_old_dev ? logp_old_dev : t->buf.logp;
+    p.adv = t->buf.adv;
+    p.mask = t->buf.mask;
+    p.terms = terms_out_dev;
+    p.J = J_out_dev;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.nodes = t->lv.offset[t->desc.T + 1];
+    p.logp_scale = static_cast<double>(logp_scale);
+    p.clip_eps = clip_eps;
+    cudaError_t e = launch_objective(p, as_stream(stream));
+    return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "objective kernel");
+}
+
+bgrpo_status bgrpo_tree_set_sde_steps(bgrpo_tree* t, const uint8_t* sde_flags_host) {
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+    uint64_t ode = 0;
+    if (sde_flags_host)
+        for (int i = 0; i < t->desc.T; ++i)
+            if (!sde_flags_host[i]) ode |= 1ull << i;
+    t->ode_bits = ode;
+    fill_coefficients(t);
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_mix_sde_steps(int32_t T, const int32_t* split_steps, int32_t n_splits, int32_t iter, int32_t window,
+                                 int32_t every, int32_t start, uint8_t* flags_out) {
+    if (T < 1 || T > BGRPO_MAX_T || !flags_out || n_splits < 0 || (n_splits > 0 && !split_steps) || iter < 0 || window < 0 || every < 1 || start < 0)
+        return fail(BGRPO_ERR_INVALID_ARG, "bad schedule arguments");
+    for (int i = 0; i < T; ++i) flags_out[i] = 0;
+    for (int q = 0; q < n_splits; ++q) {
+        if (split_steps[q] < 0 || split_steps[q] >= T) return fail(BGRPO_ERR_INVALID_ARG, "split step out of range");
+        flags_out[split_steps[q]] = 1;
+    }
+    int first = start + iter / every;
+    const int last_first = T - window > 0 ? T - window : 0;
+    if (first > last_first) first = last_first;
+    for (int j = 0; j < window && first + j < T; ++j) flags_out[first + j] = 1;
     return BGRPO_OK;
 }
 

@@ -77,6 +77,7 @@ struct bgrpo_tree {
     float t_grid[BGRPO_MAX_T + 1];
     bgrpo::StepCoef coef[BGRPO_MAX_T];
     bgrpo::LevelInfo lv;
+    uint64_t ode_bits;                   // bit i set: step i is an ODE step of the hybrid schedule (sigma = 0)
     int32_t depth;                       // steps taken so far
     int64_t D;                           // elements per node
     int32_t nchunks;                     // reward / root work items per node row
@@ -141,6 +142,12 @@ struct PruneLaunch {
     LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes, mode, k, last_split, ignore_last; uint64_t pruned_bits;
 };
 cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s);
+
+struct ObjectiveLaunch {
+    const float* logp_new; const float* logp_old; const float* adv; const uint8_t* mask; float* terms; float* J;
+    int32_t n_trees, nodes_cap, nodes; double logp_scale; float clip_eps;
+};
+cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s);
 
 // ---- MLP velocity (mlp_velocity.cu) -----------------------------------------------------------------------------
 size_t mlp_packed_bytes(int hidden);

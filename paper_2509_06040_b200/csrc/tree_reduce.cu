@@ -154,7 +154,47 @@ prune_kernel(const PruneLaunch p) {
     }
 }
 
+// Clipped GRPO objective (Eq. 5), forward value: one CTA per tree; per-thread strided sums, fixed-order reduction.
+__global__ void __launch_bounds__(kTreeThreads)
+objective_kernel(const ObjectiveLaunch p) {
+    const int tree = blockIdx.x;
+    const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    double sum = 0.0;
+    int cnt = 0;
+    for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) {
+        float term = 0.0f;
+        if (n > 0 && p.mask[row0 + n]) {
+            const double rho = exp(p.logp_scale * (static_cast<double>(p.logp_new[row0 + n]) - static_cast<double>(p.logp_old[row0 + n])));
+            const double a = static_cast<double>(p.adv[row0 + n]);
+            const double lo = 1.0 - static_cast<double>(p.clip_eps), hi = 1.0 + static_cast<double>(p.clip_eps);
+            const double t = fmin(rho * a, fmin(fmax(rho, lo), hi) * a);
+            sum += t;
+            cnt += 1;
+            term = static_cast<float>(t);
+        }
+        if (p.terms) p.terms[row0 + n] = term;
+    }
+    __shared__ double ssum[kTreeThreads / 32];
+    __shared__ int scnt[kTreeThreads / 32];
+    sum = warp_sum_d(sum);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if ((threadIdx.x & 31) == 0) { ssum[threadIdx.x >> 5] = sum; scnt[threadIdx.x >> 5] = cnt; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        int c = 0;
+        for (int w = 0; w < kTreeThreads / 32; ++w) { s += ssum[w]; c += scnt[w]; }
+        p.J[tree] = c > 0 ? static_cast<float>(s / c) : 0.0f;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s) {
+    objective_kernel<<<p.n_trees, kTreeThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
     const size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);

@@ -412,3 +412,66 @@ def test_nonfinite_reward_sets_status(B):
         B.tree_sync_status(s.tree)
     assert e.value.status == B.ERR_NONFINITE
     B.tree_sync_status(s.tree)                     # the word is cleared by the read
+
+
+# ---------------------------------------------------------------------------------------------- hybrid ODE-SDE schedule, Eq. 5
+def test_hybrid_ode_sde_rollout_and_mask(B):
+    w = Workload(name="mix", n_trees=2, tokens=600, channels=4, T=8, K=2, splits=(0, 3), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu", seed=77)
+    inp = make_inputs(w)
+    sde_steps = B.mix_sde_steps(w.T, w.splits, iteration=60, window=2, every=30, start=4)      # splits + {6, 7}
+    assert sde_steps == credit.mix_sde_steps(w.T, w.splits, 60, 2, 30, 4) == [0, 3, 6, 7]
+    s = _session(w)
+    s.upload_inputs(inp)
+    s.init()
+    B.tree_set_sde_steps(s.tree, [1 if i in sde_steps else 0 for i in range(w.T)])
+    for i in range(w.T):
+        s.step(i)
+    s.rewards()
+    s.fuse_advantage()
+    s.prune()
+    torch.cuda.synchronize()
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    grid = w.t_grid().astype(np.float64)
+    for t in range(2):
+        mu = inp.mu[t].astype(np.float64)
+        lat, logp = sde.rollout(topo, w.D, grid, f32(w.sigma), math.inf, w.seed,
+                                lambda z, i, p: sde.linear_velocity(z.astype(np.float64), float(grid[i]), mu, 0.5),
+                                tree_id=t, nodes_cap=topo.nodes, sde_steps=sde_steps)
+        assert np.abs(s.latents[t].cpu().numpy() - lat).max() <= LATENT_TOL
+        assert np.abs(s.logp[t].cpu().numpy() - logp).max() <= LOGP_TOL
+        rbar = s.rbar[t].cpu().numpy()
+        assert np.array_equal(s.mask[t].cpu().numpy(), credit.gradient_mask(topo, rbar, w.width_mode, w.width_k, (), False, sde_steps))
+    # a split on an ODE step is refused, and the default (all SDE) can be restored
+    s.init()
+    B.tree_set_sde_steps(s.tree, [0] * w.T)
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_step(s.tree, 1)
+    assert e.value.status == B.ERR_INVALID_ARG
+    B.tree_set_sde_steps(s.tree, None)
+    B.tree_step(s.tree, 1)
+    torch.cuda.synchronize()
+
+
+def test_grpo_objective_matches_oracle(B):
+    w, s, topo = _grown_session(B, 8, 2, (0, 2, 5))
+    rng = np.random.default_rng(8)
+    adv = rng.standard_normal((2, topo.nodes)).astype(np.float32)
+    mask = (rng.random((2, topo.nodes)) < 0.6).astype(np.uint8)
+    mask[1, :] = 0                                   # a tree with an empty edge set
+    old = (-np.abs(rng.standard_normal((2, topo.nodes))) - 0.2).astype(np.float32)
+    new = (old + 0.01 * rng.standard_normal((2, topo.nodes))).astype(np.float32)
+    s.adv.copy_(torch.from_numpy(adv))
+    s.mask.copy_(torch.from_numpy(mask))
+    s.logp.copy_(torch.from_numpy(old))
+    new_dev = torch.from_numpy(new).cuda()
+    J = torch.full((2,), 9.0, device="cuda")
+    terms = torch.full_like(s.logp, 9.0)
+    for eps, scale, use_buf in ((1e-4, 1.0, True), (0.2, 64.0, False)):
+        B.tree_grpo_objective(s.tree, new_dev, None if use_buf else s.logp, scale, eps, terms, J)
+        torch.cuda.synchronize()
+        for t in range(2):
+            Jr, tr = credit.grpo_objective(topo, new[t], old[t], adv[t], mask[t], f32(eps), f32(scale))
+            assert abs(J[t].item() - Jr) <= 1e-6 * max(1.0, abs(Jr))
+            assert np.abs(terms[t].cpu().numpy() - tr).max() <= 1e-6 * max(1.0, np.abs(tr).max())
+    assert J[1].item() == 0.0
