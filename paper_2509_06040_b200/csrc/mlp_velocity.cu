@@ -5,19 +5,27 @@
 //
 // One persistent CTA per SM walks 128-token tiles.  For each tile the hidden dimension is cut into chunks of 128:
 //     GEMM1(c): D1[128 tok][128 hid]  = A[128 tok][64]      * W1_c        (4 MMAs of K = 16, accumulator in TMEM)
-//     GELU     : H_c = bf16(GELU(D1))   TMEM -> registers -> shared memory (the hidden activation never leaves the SM)
-//     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, accumulator in TMEM)
+//     GELU     : H_c = bf16(2 GELU(D1))  TMEM -> registers -> TMEM: the packed bf16 activations overwrite the lower
+//                half of the columns they came from, so the hidden activation never leaves tensor memory
+//     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, A operand read from TMEM)
+// and the output tile is v = 0.5 D2 (the factor 1/2 of GELU is a power of two: taking it out of the 3072 activations
+// of a token and applying it to the 64 outputs changes no rounding).
 // Warp roles:
 //     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 3-stage ring of W1 chunks,
-//                  lane 1 a 2-stage ring of W2 chunks;
-//     warp 1       owns tensor memory; its lane 0 issues GEMM1, which runs up to three chunks ahead (D1 is
-//                  triple-buffered);
-//     warp 19      lane 0 issues GEMM2; GEMM2(c) overlaps the epilogue of chunk c + 1 (H is double-buffered);
-//     warps 2..17  GELU epilogue, four warps per TMEM lane quarter with 32 columns each, and the output tile;
+//                  lane 1 a 4-stage ring of W2 chunks;
+//     warp 1       owns tensor memory; its lane 0 issues GEMM1 into a ring of three D1 buffers; a buffer is free again
+//                  when the GEMM2 that read the activations stored in it has completed;
+//     warp 19      lane 0 issues GEMM2;
+//     warps 2..17  GELU epilogue in two groups of eight: group p takes the chunks of parity p, two warps per TMEM lane
+//                  quarter with 64 columns each.  The groups run half a period apart, so one group's
+//                  arithmetic fills the issue slots while the other hands a chunk over (barrier round trips, TMEM
+//                  load latency); a warp issues the TMEM load of its NEXT chunk before it hands the current one to
+//                  GEMM2.  All sixteen warps write the output tile (D2 is double-buffered, and a tile is written out
+//                  two chunks after its last GEMM2 was issued, when it has long completed);
 //     warp 18      converts the NEXT tile's latents to bf16 into the second A buffer while the current tile computes.
-// Operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors address; the
-// weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with one copy
-// per matrix.  No cluster multicast is used anywhere.
+// Shared-memory operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors
+// address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with
+// one copy per matrix.  No cluster multicast is used anywhere.
 //
 // Every wait is bounded (2 s): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
 // released and bit 2 of the status word is set.
@@ -30,25 +38,25 @@ constexpr int kTok = 128;                 // tokens per tile = MMA M
 constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
 constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
 constexpr int kW1Stages = 3;               // = kD1Bufs: W1 slot q is free again when GEMM1 into D1[q] has completed
-constexpr int kW2Stages = 2;               // = H buffers: W2 slot q is free again when the GEMM2 reading H[q] has completed
+constexpr int kW2Stages = 4;               // W2 slot q is free again when the GEMM2 that read it has completed
 constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 32 columns of a chunk each
 constexpr int kLoaderWarp = 2 + kEpiWarps;
 constexpr int kGemm2Warp = 3 + kEpiWarps;
 constexpr int kMlpThreads = (4 + kEpiWarps) * 32;
 constexpr uint32_t kTileBytes = kTok * 128;              // one [128 rows][128 B] operand tile = 16 KiB
 constexpr uint32_t kChunkBytes = 2 * kTileBytes;         // packed weights of a chunk: W1_c (16 KiB) then W2_c (16 KiB)
-constexpr int kD1Bufs = 3;                // GEMM1 runs two chunks ahead of the epilogue
-constexpr uint32_t kTmemCols = 512;       // D1: 3 x 128 columns, D2: 64 columns (power of two >= 448)
+constexpr int kD1Bufs = 3;                // D1(c) -> activations H(c) in place -> GEMM2(c): three chunks in flight
+constexpr uint32_t kTmemCols = 512;       // D1: 3 x 128 columns, D2: 2 x 64 columns
 constexpr uint32_t kD2Col = kD1Bufs * kHc;
+constexpr int kGroupWarps = kEpiWarps / 2; // epilogue warps that work on one chunk
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 struct MlpSmem {
     alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
     alignas(1024) unsigned char w2[kW2Stages][kTileBytes];  // W2_c as two [64 n = channel][128 B = 64 hidden] tiles
     alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
-    alignas(1024) unsigned char h[2][2][kTileBytes];        // [buffer][k half][128 tok][128 B]
-    unsigned long long w1_full[kW1Stages], w2_full[kW2Stages];
-    unsigned long long a_full[2], a_empty[2], d1_full[kD1Bufs], d1_empty[kD1Bufs], h_full[2], h_empty[2], d2_full, d2_empty;
+    unsigned long long w1_full[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
+    unsigned long long a_full[2], a_empty[2], d1_full[kD1Bufs], h_full[kD1Bufs], d1_free[kD1Bufs], d2_full[2], d2_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -103,6 +111,24 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
         else if (now - t0 > kWaitNs) { *abort_flag = 1; return false; }
     }
 }
+// True in exactly one lane of a converged warp.  Code guarded by it is known to the compiler to run in a single
+// lane, which lets the tensor-core instructions take their operands from uniform registers directly (issued under
+// `lane == 0` instead, each MMA cost about twice as many issue cycles on B200).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P1;\n\t.reg .b32 R1;\n\telect.sync R1|P1, 0xffffffff;\n\tselp.u32 %0, 1, 0, P1;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+// One non-blocking look at the barrier: 1 if the phase of the given parity is complete.
+__device__ __forceinline__ uint32_t mbar_probe(unsigned long long* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done;
+}
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, unsigned long long* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
@@ -125,6 +151,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same with the A operand in tensor memory: 128 lanes (token rows) x 8 columns, each 32-bit column holding two
+// consecutive bf16 elements of K.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // The mbarrier receives one arrival when every MMA this thread has issued so far has completed.
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -146,6 +180,29 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
           "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Waits for the thread's outstanding TMEM loads.  The destination registers of the load are named as read-write
+// operands so that every later use of them stays behind the wait.
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&r)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]),
+                   "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait32(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]),
+                   "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]),
+                   "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+                   "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -156,15 +213,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-// GELU in its tanh form on the hardware tanh: 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).  It differs from the
-// erf form by < 5e-4 absolute, below the bf16 rounding of the activation that follows.
-__device__ __forceinline__ float gelu_fast(float x) {
+// Twice the GELU in its tanh form on the hardware tanh: x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).  The tanh form
+// differs from the erf form by < 5e-4 absolute, below the bf16 rounding of the activation that follows; bf16(2a) is
+// exactly 2 bf16(a), and the output tile takes the factor back.
+__device__ __forceinline__ float gelu_x2(float x) {
     const float x2 = x * x;
     const float u = x * fmaf(x2, 0.0356774081f, 0.7978845608f);
     float th;
     asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(u));
-    const float hx = 0.5f * x;
-    return fmaf(hx, th, hx);
+    return fmaf(x, th, x);
 }
 // byte offset of the 16-byte piece `c16` of row r inside a 128-byte-swizzled tile of 128-byte rows
 __device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c16) { return r * 128u + ((c16 ^ (r & 7u)) << 4); }
@@ -192,19 +249,21 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
 
     if (threadIdx.x == 0) {
         for (int q = 0; q < kW1Stages; ++q) mbar_init(&sm.w1_full[q], 1);
-        for (int q = 0; q < kW2Stages; ++q) mbar_init(&sm.w2_full[q], 1);
+        for (int q = 0; q < kW2Stages; ++q) {
+            mbar_init(&sm.w2_full[q], 1);
+            mbar_init(&sm.w2_free[q], 1);
+        }
         for (int q = 0; q < 2; ++q) {
             mbar_init(&sm.a_full[q], 1);
             mbar_init(&sm.a_empty[q], 1);
-            mbar_init(&sm.h_full[q], kEpiWarps);
-            mbar_init(&sm.h_empty[q], 1);
+            mbar_init(&sm.d2_full[q], 1);
+            mbar_init(&sm.d2_empty[q], kEpiWarps);
         }
         for (int q = 0; q < kD1Bufs; ++q) {
             mbar_init(&sm.d1_full[q], 1);
-            mbar_init(&sm.d1_empty[q], kEpiWarps);
+            mbar_init(&sm.h_full[q], kGroupWarps);
+            mbar_init(&sm.d1_free[q], 1);
         }
-        mbar_init(&sm.d2_full, 1);
-        mbar_init(&sm.d2_empty, kEpiWarps);
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -238,7 +297,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             Ring<kW2Stages> r;
             int cc = static_cast<int>(blockIdx.x) % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
-                if (r.wrapped && !mbar_wait(&sm.h_empty[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM2 that read this slot is done
+                if (r.wrapped && !mbar_wait(&sm.w2_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM2 that read this slot is done
                 mbar_expect_tx(&sm.w2_full[r.slot], kTileBytes);
                 bulk_load(sm.w2[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes + kTileBytes, kTileBytes, &sm.w2_full[r.slot]);
                 r.advance();
@@ -247,60 +306,70 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- GEMM1 issuer
-        // Two threads issue MMAs, one per GEMM, so that a GEMM1 held back by the tensor pipe never delays the GEMM2 the
-        // epilogue is waiting for (and vice versa); completion tracking (tcgen05.commit) is per issuing thread.
-        if (lane == 0) {
-            constexpr uint32_t idesc1 = umma_idesc(kTok, kHc);
-            constexpr uint32_t kTileUnits = kTileBytes >> 4;
-            static_assert(kW1Stages == kD1Bufs, "the W1 ring and the D1 ring advance together");
-            const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]);
-            bool ok = true;
-            Ring<kD1Bufs> r;          // weights and accumulator of the next GEMM1
-            for (int it = 0; it < n_my_tiles && ok; ++it) {
-                const int ab = it & 1;
-                ok = mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag);
-                const uint32_t a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
-                for (int c = 0; c < NC && ok; ++c) {       // D1[r] = A * W1[r]
-                    ok = mbar_wait(&sm.w1_full[r.slot], r.phase, abort_flag);
-                    if (ok && r.wrapped) ok = mbar_wait(&sm.d1_empty[r.slot], r.phase ^ 1u, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t b_lo = w1_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
-                    const uint32_t d = tmem + static_cast<uint32_t>(r.slot) * kHc;
+        // Two warps issue MMAs, one per GEMM, so that a GEMM1 held back by the tensor pipe never delays the GEMM2 the
+        // epilogue is waiting for (and vice versa); completion tracking (tcgen05.commit) is per issuing thread.  The
+        // whole warp walks the loop and waits; one elected lane issues.
+        constexpr uint32_t idesc1 = umma_idesc(kTok, kHc);
+        constexpr uint32_t kTileUnits = kTileBytes >> 4;
+        static_assert(kW1Stages == kD1Bufs, "the W1 ring and the D1 ring advance together");
+        const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]);
+        bool ok = true;
+        Ring<kD1Bufs> r;          // weights and accumulator of the next GEMM1
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int ab = it & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag) ? 1 : 0) != 0;
+            const uint32_t a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
+            for (int c = 0; c < NC && ok; ++c) {       // D1[r] = A * W1[r]
+                ok = mbar_wait(&sm.w1_full[r.slot], r.phase, abort_flag);
+                if (ok && r.wrapped) ok = mbar_wait(&sm.d1_free[r.slot], r.phase ^ 1u, abort_flag);   // GEMM2 of chunk g - 3 has read its activations
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t b_lo = w1_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
+                const uint32_t d = tmem + static_cast<uint32_t>(r.slot) * kHc;
+                if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
                         umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
                     umma_commit(&sm.d1_full[r.slot]);
-                    r.advance();
                 }
-                if (ok) umma_commit(&sm.a_empty[ab]);       // every GEMM1 of this tile has been issued
+                __syncwarp();
+                r.advance();
             }
+            if (ok && elect_one()) umma_commit(&sm.a_empty[ab]);       // every GEMM1 of this tile has been issued
+            __syncwarp();
         }
     } else if (warp == kGemm2Warp) {
         // ---------------------------------------------------------------- GEMM2 issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc2 = umma_idesc(kTok, kCh);
-            constexpr uint32_t kTileUnits = kTileBytes >> 4;
-            const uint32_t w2_lo = desc_lo(sm.w2[0]), h_lo = desc_lo(sm.h[0][0]);
-            bool ok = true;
-            Ring<2> r;                // H buffer and weights of the next GEMM2
-            for (int it = 0; it < n_my_tiles && ok; ++it) {
-                for (int c = 0; c < NC && ok; ++c) {       // D2 += H[r] * W2[r]
-                    ok = mbar_wait(&sm.w2_full[r.slot], r.phase, abort_flag);
-                    if (ok) ok = mbar_wait(&sm.h_full[r.slot], r.phase, abort_flag);
-                    if (ok && c == 0 && it > 0) ok = mbar_wait(&sm.d2_empty, static_cast<uint32_t>(it - 1) & 1u, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t ha_lo = h_lo + static_cast<uint32_t>(r.slot) * (2u * kTileUnits);
-                    const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
+        constexpr uint32_t idesc2 = umma_idesc(kTok, kCh);
+        constexpr uint32_t kTileUnits = kTileBytes >> 4;
+        const uint32_t w2_lo = desc_lo(sm.w2[0]);
+        bool ok = true;
+        Ring<kD1Bufs> rh;         // D1 buffer holding the activations of the next GEMM2
+        Ring<kW2Stages> rw;       // its weights
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            for (int c = 0; c < NC && ok; ++c) {       // D2 += H[rh] * W2[rw]
+                ok = mbar_wait(&sm.w2_full[rw.slot], rw.phase, abort_flag);
+                if (ok) ok = mbar_wait(&sm.h_full[rh.slot], rh.phase, abort_flag);
+                if (ok && c == 0 && it >= 2)      // the tile that used this D2 buffer two tiles ago has been written out
+                    ok = mbar_wait(&sm.d2_empty[it & 1], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t h_col = tmem + static_cast<uint32_t>(rh.slot) * kHc;
+                const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(rw.slot) * kTileUnits;
+                if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < kHc / 16; ++k)
-                        umma_bf16(tmem + kD2Col, desc64(ha_lo + (k / 4) * kTileUnits + 2u * (k % 4)),
-                                  desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&sm.h_empty[r.slot]);
-                    if (c == NC - 1) umma_commit(&sm.d2_full);
-                    r.advance();
+                    for (int k = 0; k < kHc / 16; ++k)      // hidden 16k .. 16k+15 of the chunk: 8 packed columns at 32 (k/2) + 8 (k%2)
+                        umma_bf16_ts(tmem + kD2Col + static_cast<uint32_t>(it & 1) * kCh, h_col + 32u * (k / 2) + 8u * (k % 2),
+                                     desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&sm.d1_free[rh.slot]);
+                    umma_commit(&sm.w2_free[rw.slot]);
+                    if (c == NC - 1) umma_commit(&sm.d2_full[it & 1]);
                 }
+                __syncwarp();
+                rh.advance();
+                rw.advance();
             }
         }
     } else if (warp == kLoaderWarp) {
@@ -342,65 +411,89 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int ew = warp - 2;                  // 0..15
+        const int group = ew >> 3;                // parity of the chunks this warp works on
         const uint32_t quarter = static_cast<uint32_t>(warp & 3);   // TMEM lanes this warp may touch: 32*quarter .. +31
-        const uint32_t sub = static_cast<uint32_t>(ew >> 2);        // which 32 of the chunk's 128 columns
+        const uint32_t sub = static_cast<uint32_t>(ew >> 2) & 3u;   // output tile: which 16 of the 64 channels
         const uint32_t row = quarter * 32u + static_cast<uint32_t>(lane);       // token row of this thread in the tile
         const uint32_t lane_addr = (quarter * 32u) << 16;
+        const uint32_t slice = tmem + lane_addr + (sub & 1u) * 64u; // this warp's 64 columns inside a D1 buffer
         bool ok = true;
-        Ring<kD1Bufs> rd1;
-        Ring<2> rh;
-        for (int it = 0; it < n_my_tiles && ok; ++it) {
-            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
-            for (int c = 0; c < NC && ok; ++c) {
-                ok = mbar_wait(&sm.d1_full[rd1.slot], rd1.phase, abort_flag);
-                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;      // keep every verdict warp-uniform: the TMEM loads are warp-wide
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t acc[32];
-                tmem_ld32(tmem + lane_addr + static_cast<uint32_t>(rd1.slot) * kHc + sub * 32u, acc);
-                tmem_ld_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.d1_empty[rd1.slot]);      // D1 is in registers: a later GEMM1 may overwrite it
-                rd1.advance();
-                if (rh.wrapped) ok = mbar_wait(&sm.h_empty[rh.slot], rh.phase ^ 1u, abort_flag);      // GEMM2 of chunk c - 2 has read this H buffer
-                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
-                if (!ok) break;
-                unsigned char* htile = sm.h[rh.slot][sub >> 1];    // hidden columns 0..63 / 64..127 are the two K halves of GEMM2
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {                      // 8 columns -> one 16-byte piece
-                    uint4 piece;
-                    piece.x = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 0])), gelu_fast(__uint_as_float(acc[8 * j + 1])));
-                    piece.y = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 2])), gelu_fast(__uint_as_float(acc[8 * j + 3])));
-                    piece.z = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 4])), gelu_fast(__uint_as_float(acc[8 * j + 5])));
-                    piece.w = pack_bf16(gelu_fast(__uint_as_float(acc[8 * j + 6])), gelu_fast(__uint_as_float(acc[8 * j + 7])));
-                    *reinterpret_cast<uint4*>(htile + sw128(row, (sub & 1u) * 4u + static_cast<uint32_t>(j))) = piece;
-                }
-                proxy_fence();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.h_full[rh.slot]);
-                rh.advance();
-            }
-            if (!ok) break;
-            // ---- output tile: D2 -> v (this warp's 16 of the 64 channels)
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d2_full, static_cast<uint32_t>(it) & 1u, abort_flag) ? 1 : 0) != 0;
-            if (!ok) break;
+        int next_out = 0;             // first tile this warp has not written out yet
+
+        // v = 0.5 D2 of tile t (this warp's 32 rows x 16 channels)
+        auto output_tile = [&](int t) -> bool {
+            const int b = t & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(&sm.d2_full[b], static_cast<uint32_t>(t >> 1) & 1u, abort_flag) ? 1 : 0)) return false;
             tc_fence_after();
             uint32_t out[16];
-            tmem_ld16(tmem + lane_addr + kD2Col + sub * 16u, out);
-            tmem_ld_wait();
+            tmem_ld16(tmem + lane_addr + kD2Col + static_cast<uint32_t>(b) * kCh + sub * 16u, out);
+            tmem_ld_wait16(out);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.d2_empty);
-            const int64_t q = tok0 + row;
+            if (lane == 0) mbar_arrive(&sm.d2_empty[b]);
+            const int64_t q = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(t) * gridDim.x) * kTok + row;
             if (q < p.n_tokens) {
                 float4* dst = reinterpret_cast<float4*>(p.v_out + q * kCh + sub * 16u);
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    dst[j] = make_float4(__uint_as_float(out[4 * j]), __uint_as_float(out[4 * j + 1]), __uint_as_float(out[4 * j + 2]),
-                                         __uint_as_float(out[4 * j + 3]));
+                    dst[j] = make_float4(0.5f * __uint_as_float(out[4 * j]), 0.5f * __uint_as_float(out[4 * j + 1]),
+                                         0.5f * __uint_as_float(out[4 * j + 2]), 0.5f * __uint_as_float(out[4 * j + 3]));
+            }
+            return true;
+        };
+        // 32 accumulator columns -> 16 columns of packed bf16 activations, written over the first half of their source
+        auto activate = [&](uint32_t (&acc)[32], uint32_t taddr) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int m = 0; m < 16; ++m)
+                pk[m] = pack_bf16(gelu_x2(__uint_as_float(acc[2 * m])), gelu_x2(__uint_as_float(acc[2 * m + 1])));
+            tmem_st16(taddr, pk);
+        };
+
+        uint32_t acc[32];
+        int g = group;                // chunk index within this CTA's sequence of tiles x chunks
+        if (g < n_my_chunks) {        // first 32 columns of the first chunk
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[g % kD1Bufs], static_cast<uint32_t>(g / kD1Bufs) & 1u, abort_flag) ? 1 : 0) != 0;
+            if (ok) {
+                tc_fence_after();
+                tmem_ld32(slice + static_cast<uint32_t>(g % kD1Bufs) * kHc, acc);
+                tmem_ld_wait32(acc);
             }
         }
+        for (; g < n_my_chunks && ok; g += 2) {
+            // tiles whose last GEMM2 was issued at least two chunks ago
+            while (ok && (next_out + 1) * NC + 2 <= g) ok = output_tile(next_out++);
+            if (!ok) break;
+            const int slot = g % kD1Bufs;
+            const uint32_t base = slice + static_cast<uint32_t>(slot) * kHc;
+            activate(acc, base);                              // acc holds columns 0..31 of this warp's 64
+            tmem_ld32(base + 32u, acc);
+            // look at the next chunk's barrier now; the answer is used after the arithmetic
+            const int gn = g + 2;
+            const bool more = gn < n_my_chunks;
+            const int nslot = gn % kD1Bufs;
+            const uint32_t nphase = static_cast<uint32_t>(gn / kD1Bufs) & 1u;
+            uint32_t next_ready = 1u;
+            if (more) next_ready = mbar_probe(&sm.d1_full[nslot], nphase);
+            tmem_ld_wait32(acc);
+            activate(acc, base + 32u);                        // columns 32..63
+            if (more) {
+                if (!__all_sync(0xffffffffu, next_ready))
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[nslot], nphase, abort_flag) ? 1 : 0) != 0;
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld32(slice + static_cast<uint32_t>(nslot) * kHc, acc);      // in flight during the hand-over below
+                }
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.h_full[slot]);
+            if (more && ok) tmem_ld_wait32(acc);
+        }
+        while (ok && next_out < n_my_tiles) ok = output_tile(next_out++);
+        tmem_ld_wait();
+        tmem_st_wait();
     }
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
