@@ -5,24 +5,26 @@
 //
 // One persistent CTA per SM walks 128-token tiles.  For each tile the hidden dimension is cut into chunks of 128:
 //     GEMM1(c): D1[128 tok][128 hid]  = A[128 tok][64]      * W1_c        (4 MMAs of K = 16, accumulator in TMEM)
-//     GELU     : H_c = bf16(2 GELU(D1))  TMEM -> registers -> TMEM: the packed bf16 activations overwrite the lower
-//                half of the columns they came from, so the hidden activation never leaves tensor memory
+//     GELU     : H_c = bf16(2 GELU(D1))  TMEM -> registers -> TMEM (64 columns of packed bf16 pairs): the hidden
+//                activation never leaves tensor memory
 //     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, A operand read from TMEM)
 // and the output tile is v = 0.5 D2 (the factor 1/2 of GELU is a power of two: taking it out of the 3072 activations
 // of a token and applying it to the 64 outputs changes no rounding).
 // Warp roles:
 //     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 3-stage ring of W1 chunks,
 //                  lane 1 a 4-stage ring of W2 chunks;
-//     warp 1       owns tensor memory; its lane 0 issues GEMM1 into a ring of three D1 buffers; a buffer is free again
-//                  when the GEMM2 that read the activations stored in it has completed;
-//     warp 19      lane 0 issues GEMM2;
+//     warp 1       owns tensor memory and issues GEMM1; D1 has one buffer per chunk parity, free again as soon as the
+//                  epilogue group of that parity has loaded it, so GEMM1(c + 2) runs during the epilogue of chunk c;
+//     warp 19      issues GEMM2 from the activation buffer of the chunk's parity;
 //     warps 2..17  GELU epilogue in two groups of eight: group p takes the chunks of parity p, two warps per TMEM lane
 //                  quarter with 64 columns each.  The groups run half a period apart, so one group's
 //                  arithmetic fills the issue slots while the other hands a chunk over (barrier round trips, TMEM
 //                  load latency); a warp issues the TMEM load of its NEXT chunk before it hands the current one to
 //                  GEMM2.  All sixteen warps write the output tile (D2 is double-buffered, and a tile is written out
 //                  two chunks after its last GEMM2 was issued, when it has long completed);
-//     warp 18      converts the NEXT tile's latents to bf16 into the second A buffer while the current tile computes.
+//     warp 18      brings the NEXT tile's latents in with bulk asynchronous copies (one per tree the tile touches) into
+//                  a float32 staging buffer and converts them to the bf16 A tile while the current tile computes.  (Plain
+//                  loads from one warp kept only 4 KiB in flight and took longer per tile than the arithmetic.)
 // Shared-memory operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors
 // address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with
 // one copy per matrix.  No cluster multicast is used anywhere.
@@ -37,7 +39,7 @@ namespace {
 constexpr int kTok = 128;                 // tokens per tile = MMA M
 constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
 constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
-constexpr int kW1Stages = 3;               // = kD1Bufs: W1 slot q is free again when GEMM1 into D1[q] has completed
+constexpr int kW1Stages = 3;               // W1 slot q is free again when the GEMM1 that read it has completed
 constexpr int kW2Stages = 4;               // W2 slot q is free again when the GEMM2 that read it has completed
 constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 32 columns of a chunk each
 constexpr int kLoaderWarp = 2 + kEpiWarps;
@@ -45,9 +47,9 @@ constexpr int kGemm2Warp = 3 + kEpiWarps;
 constexpr int kMlpThreads = (4 + kEpiWarps) * 32;
 constexpr uint32_t kTileBytes = kTok * 128;              // one [128 rows][128 B] operand tile = 16 KiB
 constexpr uint32_t kChunkBytes = 2 * kTileBytes;         // packed weights of a chunk: W1_c (16 KiB) then W2_c (16 KiB)
-constexpr int kD1Bufs = 3;                // D1(c) -> activations H(c) in place -> GEMM2(c): three chunks in flight
-constexpr uint32_t kTmemCols = 512;       // D1: 3 x 128 columns, D2: 2 x 64 columns
-constexpr uint32_t kD2Col = kD1Bufs * kHc;
+constexpr uint32_t kTmemCols = 512;       // D1: 2 x 128 columns, H: 2 x 64, D2: 2 x 64; index = chunk parity (D1, H) or tile parity (D2)
+constexpr uint32_t kHCol = 2 * kHc;
+constexpr uint32_t kD2Col = kHCol + 2 * (kHc / 2);
 constexpr int kGroupWarps = kEpiWarps / 2; // epilogue warps that work on one chunk
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
@@ -55,8 +57,9 @@ struct MlpSmem {
     alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
     alignas(1024) unsigned char w2[kW2Stages][kTileBytes];  // W2_c as two [64 n = channel][128 B = 64 hidden] tiles
     alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
-    unsigned long long w1_full[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
-    unsigned long long a_full[2], a_empty[2], d1_full[kD1Bufs], h_full[kD1Bufs], d1_free[kD1Bufs], d2_full[2], d2_empty[2];
+    alignas(1024) float stage[kTok * kCh];                   // float32 latents of the next tile, as they are in global memory
+    unsigned long long w1_full[kW1Stages], w1_free[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
+    unsigned long long stage_full, a_full[2], a_empty[2], d1_full[2], d1_empty[2], h_full[2], h_free[2], d2_full[2], d2_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -248,21 +251,24 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     volatile int* abort_flag = &sm.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int q = 0; q < kW1Stages; ++q) mbar_init(&sm.w1_full[q], 1);
+        for (int q = 0; q < kW1Stages; ++q) {
+            mbar_init(&sm.w1_full[q], 1);
+            mbar_init(&sm.w1_free[q], 1);
+        }
         for (int q = 0; q < kW2Stages; ++q) {
             mbar_init(&sm.w2_full[q], 1);
             mbar_init(&sm.w2_free[q], 1);
         }
+        mbar_init(&sm.stage_full, 1);
         for (int q = 0; q < 2; ++q) {
             mbar_init(&sm.a_full[q], 1);
             mbar_init(&sm.a_empty[q], 1);
             mbar_init(&sm.d2_full[q], 1);
             mbar_init(&sm.d2_empty[q], kEpiWarps);
-        }
-        for (int q = 0; q < kD1Bufs; ++q) {
             mbar_init(&sm.d1_full[q], 1);
+            mbar_init(&sm.d1_empty[q], kGroupWarps);
             mbar_init(&sm.h_full[q], kGroupWarps);
-            mbar_init(&sm.d1_free[q], 1);
+            mbar_init(&sm.h_free[q], 1);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -287,7 +293,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             Ring<kW1Stages> r;
             int cc = static_cast<int>(blockIdx.x) % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
-                if (r.wrapped && !mbar_wait(&sm.d1_full[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM1 that read this slot is done
+                if (r.wrapped && !mbar_wait(&sm.w1_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM1 that read this slot is done
                 mbar_expect_tx(&sm.w1_full[r.slot], kTileBytes);
                 bulk_load(sm.w1[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes, kTileBytes, &sm.w1_full[r.slot]);
                 r.advance();
@@ -311,27 +317,29 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         // whole warp walks the loop and waits; one elected lane issues.
         constexpr uint32_t idesc1 = umma_idesc(kTok, kHc);
         constexpr uint32_t kTileUnits = kTileBytes >> 4;
-        static_assert(kW1Stages == kD1Bufs, "the W1 ring and the D1 ring advance together");
         const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]);
         bool ok = true;
-        Ring<kD1Bufs> r;          // weights and accumulator of the next GEMM1
+        Ring<kW1Stages> r;        // weights of the next GEMM1
+        int g = 0;                // chunks issued so far: D1 buffer g & 1, its use number g >> 1
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int ab = it & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag) ? 1 : 0) != 0;
             const uint32_t a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
-            for (int c = 0; c < NC && ok; ++c) {       // D1[r] = A * W1[r]
+            for (int c = 0; c < NC && ok; ++c, ++g) {       // D1[g & 1] = A * W1[r]
                 ok = mbar_wait(&sm.w1_full[r.slot], r.phase, abort_flag);
-                if (ok && r.wrapped) ok = mbar_wait(&sm.d1_free[r.slot], r.phase ^ 1u, abort_flag);   // GEMM2 of chunk g - 3 has read its activations
+                if (ok && g >= 2)      // the epilogue group of this parity has loaded chunk g - 2
+                    ok = mbar_wait(&sm.d1_empty[g & 1], static_cast<uint32_t>((g >> 1) - 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t b_lo = w1_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
-                const uint32_t d = tmem + static_cast<uint32_t>(r.slot) * kHc;
+                const uint32_t d = tmem + static_cast<uint32_t>(g & 1) * kHc;
                 if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
                         umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
-                    umma_commit(&sm.d1_full[r.slot]);
+                    umma_commit(&sm.d1_full[g & 1]);
+                    umma_commit(&sm.w1_free[r.slot]);
                 }
                 __syncwarp();
                 r.advance();
@@ -345,68 +353,79 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         constexpr uint32_t kTileUnits = kTileBytes >> 4;
         const uint32_t w2_lo = desc_lo(sm.w2[0]);
         bool ok = true;
-        Ring<kD1Bufs> rh;         // D1 buffer holding the activations of the next GEMM2
-        Ring<kW2Stages> rw;       // its weights
+        Ring<kW2Stages> rw;       // weights of the next GEMM2
+        int g = 0;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            for (int c = 0; c < NC && ok; ++c) {       // D2 += H[rh] * W2[rw]
+            for (int c = 0; c < NC && ok; ++c, ++g) {       // D2 += H[g & 1] * W2[rw]
                 ok = mbar_wait(&sm.w2_full[rw.slot], rw.phase, abort_flag);
-                if (ok) ok = mbar_wait(&sm.h_full[rh.slot], rh.phase, abort_flag);
+                if (ok) ok = mbar_wait(&sm.h_full[g & 1], static_cast<uint32_t>(g >> 1) & 1u, abort_flag);
                 if (ok && c == 0 && it >= 2)      // the tile that used this D2 buffer two tiles ago has been written out
                     ok = mbar_wait(&sm.d2_empty[it & 1], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t h_col = tmem + static_cast<uint32_t>(rh.slot) * kHc;
+                const uint32_t h_col = tmem + kHCol + static_cast<uint32_t>(g & 1) * (kHc / 2);
                 const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(rw.slot) * kTileUnits;
                 if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < kHc / 16; ++k)      // hidden 16k .. 16k+15 of the chunk: 8 packed columns at 32 (k/2) + 8 (k%2)
-                        umma_bf16_ts(tmem + kD2Col + static_cast<uint32_t>(it & 1) * kCh, h_col + 32u * (k / 2) + 8u * (k % 2),
+                    for (int k = 0; k < kHc / 16; ++k)      // hidden 16k .. 16k+15 of the chunk: packed columns 8k .. 8k+7
+                        umma_bf16_ts(tmem + kD2Col + static_cast<uint32_t>(it & 1) * kCh, h_col + 8u * k,
                                      desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&sm.d1_free[rh.slot]);
+                    umma_commit(&sm.h_free[g & 1]);
                     umma_commit(&sm.w2_free[rw.slot]);
                     if (c == NC - 1) umma_commit(&sm.d2_full[it & 1]);
                 }
                 __syncwarp();
-                rh.advance();
                 rw.advance();
             }
         }
     } else if (warp == kLoaderWarp) {
-        // ---------------------------------------------------------------- latent tile -> bf16, K-major swizzled
-        // The warp covers 2 rows per step (16 lanes x 16 B per row); 8 steps are in flight at a time.
+        // ---------------------------------------------------------------- latent tile -> staging -> bf16, K-major swizzled
+        // Tokens of the frontier are numbered tree by tree; the rows of one tree are contiguous in the pool, so a tile is
+        // one copy per tree it touches.  Rows past the last token keep whatever the staging buffer held: a row of A
+        // only feeds the same row of the output, which is not written.
+        auto issue_tile_copy = [&](int it) {       // one lane
+            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
+            int64_t remaining = p.n_tokens - tok0;
+            if (remaining > kTok) remaining = kTok;
+            mbar_expect_tx(&sm.stage_full, static_cast<uint32_t>(remaining) * (kCh * 4u));
+            int64_t q = tok0;
+            float* dst = sm.stage;
+            while (remaining > 0) {
+                const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
+                int64_t seg = p.tokens_per_tree - rr;
+                if (seg > remaining) seg = remaining;
+                bulk_load(dst, p.latents + tree * p.tree_stride + p.row_offset + rr * kCh, static_cast<uint32_t>(seg) * (kCh * 4u), &sm.stage_full);
+                dst += seg * kCh;
+                q += seg;
+                remaining -= seg;
+            }
+        };
         bool ok = true;
+        if (n_my_tiles > 0 && lane == 0) issue_tile_copy(0);
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int ab = it & 1;
-            if (it >= 2) ok = mbar_wait(&sm.a_empty[ab], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
+            ok = mbar_wait(&sm.stage_full, static_cast<uint32_t>(it) & 1u, abort_flag);
+            if (ok && it >= 2) ok = mbar_wait(&sm.a_empty[ab], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
             ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
             if (!ok) break;
-            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
-            const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row
+            const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row; the warp covers 2 rows per step
             unsigned char* atile = sm.a[ab];
-            for (int r0 = 0; r0 < kTok; r0 += 16) {
-                float4 zv[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int64_t q = tok0 + r0 + 2 * u + (lane >> 4);
-                    zv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (q < p.n_tokens) {
-                        const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
-                        zv[u] = __ldcs(reinterpret_cast<const float4*>(p.latents + tree * p.tree_stride + p.row_offset + rr * kCh) + c4);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t r = static_cast<uint32_t>(r0 + 2 * u + (lane >> 4));
-                    uint2 packed2;
-                    packed2.x = pack_bf16(zv[u].x, zv[u].y);
-                    packed2.y = pack_bf16(zv[u].z, zv[u].w);
-                    *reinterpret_cast<uint2*>(atile + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
-                }
+#pragma unroll 8
+            for (int r0 = 0; r0 < kTok; r0 += 2) {
+                const uint32_t r = static_cast<uint32_t>(r0 + (lane >> 4));
+                const float4 zv = *reinterpret_cast<const float4*>(sm.stage + r * kCh + c4 * 4u);
+                uint2 packed2;
+                packed2.x = pack_bf16(zv.x, zv.y);
+                packed2.y = pack_bf16(zv.z, zv.w);
+                *reinterpret_cast<uint2*>(atile + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
             }
             proxy_fence();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.a_full[ab]);
+            if (lane == 0) {
+                mbar_arrive(&sm.a_full[ab]);
+                if (it + 1 < n_my_tiles) issue_tile_copy(it + 1);      // every lane has read the staging buffer
+            }
         }
     } else {
         // ---------------------------------------------------------------- epilogue warps
@@ -416,7 +435,6 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         const uint32_t sub = static_cast<uint32_t>(ew >> 2) & 3u;   // output tile: which 16 of the 64 channels
         const uint32_t row = quarter * 32u + static_cast<uint32_t>(lane);       // token row of this thread in the tile
         const uint32_t lane_addr = (quarter * 32u) << 16;
-        const uint32_t slice = tmem + lane_addr + (sub & 1u) * 64u; // this warp's 64 columns inside a D1 buffer
         bool ok = true;
         int next_out = 0;             // first tile this warp has not written out yet
 
@@ -441,22 +459,22 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             }
             return true;
         };
-        // 32 accumulator columns -> 16 columns of packed bf16 activations, written over the first half of their source
-        auto activate = [&](uint32_t (&acc)[32], uint32_t taddr) {
-            uint32_t pk[16];
+        // 32 accumulator columns -> 16 registers of packed bf16 activation pairs
+        auto activate = [&](const uint32_t (&acc)[32], uint32_t (&pk)[16]) {
 #pragma unroll
             for (int m = 0; m < 16; ++m)
                 pk[m] = pack_bf16(gelu_x2(__uint_as_float(acc[2 * m])), gelu_x2(__uint_as_float(acc[2 * m + 1])));
-            tmem_st16(taddr, pk);
         };
+        const uint32_t d1_slice = tmem + lane_addr + static_cast<uint32_t>(group) * kHc + (sub & 1u) * 64u;              // 64 fp32 columns
+        const uint32_t h_slice = tmem + lane_addr + kHCol + static_cast<uint32_t>(group) * (kHc / 2) + (sub & 1u) * 32u;  // 32 packed columns
 
-        uint32_t acc[32];
-        int g = group;                // chunk index within this CTA's sequence of tiles x chunks
+        uint32_t acc[32], pk[16];
+        int g = group;                // chunk index within this CTA's sequence of tiles x chunks; use number g >> 1 of the buffers
         if (g < n_my_chunks) {        // first 32 columns of the first chunk
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[g % kD1Bufs], static_cast<uint32_t>(g / kD1Bufs) & 1u, abort_flag) ? 1 : 0) != 0;
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], 0u, abort_flag) ? 1 : 0) != 0;
             if (ok) {
                 tc_fence_after();
-                tmem_ld32(slice + static_cast<uint32_t>(g % kD1Bufs) * kHc, acc);
+                tmem_ld32(d1_slice, acc);
                 tmem_ld_wait32(acc);
             }
         }
@@ -464,32 +482,37 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             // tiles whose last GEMM2 was issued at least two chunks ago
             while (ok && (next_out + 1) * NC + 2 <= g) ok = output_tile(next_out++);
             if (!ok) break;
-            const int slot = g % kD1Bufs;
-            const uint32_t base = slice + static_cast<uint32_t>(slot) * kHc;
-            activate(acc, base);                              // acc holds columns 0..31 of this warp's 64
-            tmem_ld32(base + 32u, acc);
-            // look at the next chunk's barrier now; the answer is used after the arithmetic
-            const int gn = g + 2;
-            const bool more = gn < n_my_chunks;
-            const int nslot = gn % kD1Bufs;
-            const uint32_t nphase = static_cast<uint32_t>(gn / kD1Bufs) & 1u;
-            uint32_t next_ready = 1u;
-            if (more) next_ready = mbar_probe(&sm.d1_full[nslot], nphase);
-            tmem_ld_wait32(acc);
-            activate(acc, base + 32u);                        // columns 32..63
-            if (more) {
-                if (!__all_sync(0xffffffffu, next_ready))
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[nslot], nphase, abort_flag) ? 1 : 0) != 0;
-                if (ok) {
-                    tc_fence_after();
-                    tmem_ld32(slice + static_cast<uint32_t>(nslot) * kHc, acc);      // in flight during the hand-over below
-                }
+            const uint32_t use = static_cast<uint32_t>(g >> 1);
+            // is the GEMM2 that read this group's previous activations done?  (asked now, needed after the arithmetic)
+            uint32_t h_ready = 1u;
+            if (g >= 2) h_ready = mbar_probe(&sm.h_free[group], (use - 1u) & 1u);
+            activate(acc, pk);                                // columns 0..31 of this warp's 64
+            tmem_ld32(d1_slice + 32u, acc);                   // columns 32..63, in flight during the store below
+            if (!__all_sync(0xffffffffu, h_ready))
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.h_free[group], (use - 1u) & 1u, abort_flag) ? 1 : 0) != 0;
+            if (ok) {
+                tc_fence_after();
+                tmem_st16(h_slice, pk);
             }
+            tmem_ld_wait32(acc);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.d1_empty[group]);  // D1 of this chunk is in registers: GEMM1 of chunk g + 2 may go
+            if (!ok) break;
+            activate(acc, pk);
+            tmem_st16(h_slice + 16u, pk);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.h_full[slot]);
-            if (more && ok) tmem_ld_wait32(acc);
+            if (lane == 0) mbar_arrive(&sm.h_full[group]);
+            if (g + 2 < n_my_chunks) {                        // first half of the next chunk
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], (use + 1u) & 1u, abort_flag) ? 1 : 0) != 0;
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld32(d1_slice, acc);
+                    tmem_ld_wait32(acc);
+                }
+            }
         }
         while (ok && next_out < n_my_tiles) ok = output_tile(next_out++);
         tmem_ld_wait();
