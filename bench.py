@@ -44,8 +44,8 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_TRAFFIC = {
     "step_kernel": {"workload": "video", "bytes": 75.599104e6 + 12.592896e6, "units": 8 * 2096640,
                     "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "d6ef704e319c"},
-    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.249216e6 + 212.080384e6, "units": 1036800,
-                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "ca53c8c3093c"},
+    "mlp_velocity_kernel": {"workload": "8 image-shaped trees, frontier width 16", "bytes": 67.183616e6 + 15.853056e6,
+                            "units": 259200, "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "d8e9e9052c8b"},
 }
 
 
@@ -289,10 +289,17 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
         fl = np.array(mlp_flops_per_launch(w, w.n_trees), dtype=np.float64)
         tf = fl.sum() / (t_mlp.sum() * 1e-3) / 1e12
         peak_tf = float(peaks["bf16_tflops"])
+        # one hardware tanh per hidden activation: the XU pipe issues 16 per clock per SM
+        sms = torch.cuda.get_device_properties(s.device).multi_processor_count
+        xu_peak = 16.0 * sms * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6
+        tanh_rate = fl.sum() / (4.0 * w.channels) / (t_mlp.sum() * 1e-3)
         roof = {"bound": "tensor", "kernel": "mlp_velocity_kernel", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": tf / peak_tf, "peak_source": peaks["_source"], "launches_per_pass": w.T,
                 "flops_per_pass": float(fl.sum()), "ms_per_pass": float(t_mlp.sum()),
-                "note": "the stage is bound by the GELU epilogue on the ordinary ALUs, not by the tensor pipe",
+                "note": "a dense contraction, so reported against the tensor peak; the pipe that binds it is the XU "
+                        "(one hardware tanh per hidden activation), see xu_bound",
+                "xu_bound": {"bound": "alu", "unit": "Gtanh/s", "achieved": tanh_rate / 1e9, "peak": xu_peak / 1e9,
+                             "frac": tanh_rate / xu_peak, "peak_source": "16 tanh/clk/SM x SMs x max SM clock"},
                 "traffic": ncu_traffic("mlp_velocity_kernel", float(w.n_trees * w.model_evals * w.tokens) / w.T)}
     return roof, roof_step, breakdown
 
