@@ -139,6 +139,17 @@ bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* tree, const float* mu_dev, f
  * Errors: STATE (already at depth T; NULL v_dev without a bound velocity), CAPACITY (children exceed nodes_cap), CUDA. */
 bgrpo_status bgrpo_tree_step(bgrpo_tree* tree, int32_t split_flag, const float* v_dev, void* stream);
 
+/* tree_rollout_fused: all T steps of tree_step in one launch, for the bound closed-form velocity (Branch Rollout
+ * Algorithm: "reusing shared prefixes"; Eq. 2; Algorithm 1 "Build rollout tree").  That velocity acts on every latent
+ * element by itself, so one thread can carry its elements from the root to every leaf, depth first, and write each
+ * node once: nothing is read back between depths.  Call it on a freshly initialised or reset tree.  split_flags_host:
+ * host array of T flags, non-zero = step i forks every node into K children.  Latents, node table and log-probs are the
+ * ones T calls of tree_step give (latents and table bit for bit; log-probs up to the order of a float32 partial sum),
+ * and buffers.logp is final when the call's kernels have run.  At most 6 split steps.
+ * Errors: STATE (tree not at depth 0, no bound linear velocity), CAPACITY (tree exceeds nodes_cap), UNSUPPORTED (more
+ * than 6 split steps: use tree_step), INVALID_ARG (a split on an ODE step of the hybrid schedule), CUDA. */
+bgrpo_status bgrpo_tree_rollout_fused(bgrpo_tree* tree, const uint8_t* split_flags_host, void* stream);
+
 /* tree_logprob: log pi(z_child | z_parent) of stored edges under a GIVEN velocity (the numerator of rho_e in Eq. 5;
  * under the behaviour velocity it reproduces the step-time values, the summands of s_l in Eq. 3).
  * step >= 0: the edges of that step, v_dev = device [n_trees][W_step][D] or NULL (bound linear velocity).

@@ -49,7 +49,7 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     size_t b = kScratchHeader;
     b += ((static_cast<size_t>(rows) * sizeof(unsigned int) + 255) / 256) * 256;
     b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
-    b += static_cast<size_t>(rows) * nchunks_step_of(D) * kStepWarps * sizeof(float);
+    b += static_cast<size_t>(rows) * static_cast<size_t>(partials_per_row(D)) * sizeof(float);
     return b;
 }
 
@@ -285,6 +285,70 @@ bgrpo_status bgrpo_tree_step(bgrpo_tree* t, int32_t split_flag, const float* v_d
     t->lv.width[i + 1] = static_cast<int32_t>(W_out);
     t->lv.offset[i + 2] = static_cast<int32_t>(off_out + W_out);
     t->depth = i + 1;
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_rollout_fused(bgrpo_tree* t, const uint8_t* split_flags_host, void* stream) {
+    if (!t || !split_flags_host) return fail(BGRPO_ERR_INVALID_ARG, "tree or split_flags is NULL");
+    if (t->depth != 0) return fail(BGRPO_ERR_STATE, "the whole-tree rollout starts from a freshly initialised or reset tree");
+    if (!t->mu) return fail(BGRPO_ERR_STATE, "the whole-tree rollout needs the bound closed-form velocity");
+    const int T = t->desc.T;
+    FusedLaunch p;
+    std::memset(&p, 0, sizeof(p));
+    int n_splits = 0;
+    int64_t width = 1, off = 1;
+    p.off[0] = 0;
+    p.off[1] = 1;
+    for (int i = 0; i < T; ++i) {
+        const bool split = split_flags_host[i] != 0;
+        if (split) {
+            if (((t->ode_bits >> i) & 1ull) && t->desc.sigma > 0.0f)
+                return fail(BGRPO_ERR_INVALID_ARG, "a split step must be an SDE step of the hybrid schedule");
+            ++n_splits;
+            p.split_bits |= 1ull << i;
+            width *= t->desc.K;
+        }
+        off += width;
+        if (off > t->desc.nodes_cap) return fail(BGRPO_ERR_CAPACITY, "children exceed nodes_cap");
+        p.off[i + 2] = static_cast<int32_t>(off);
+        const StepCoef& k = t->coef[i];
+        p.ca[i] = k.lin_a;
+        p.cb[i] = k.lin_b;
+        p.g[i] = k.g;
+        p.inv_2g2[i] = k.inv_2g2;
+        p.logp_const[i] = k.logp_const;
+    }
+    if (n_splits > kFusedMaxSplits) return fail(BGRPO_ERR_UNSUPPORTED, "more split steps than the whole-tree kernel walks; use tree_step");
+    p.latents = t->buf.latents;
+    p.mu = t->mu;
+    p.logp = t->buf.logp;
+    p.table = t->buf.node_table;
+    p.partialsf = t->partialsf;
+    p.D = t->D;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.nchunks = static_cast<int32_t>((t->D / 4 + kFusedChunkVec - 1) / kFusedChunkVec);
+    p.per_row = static_cast<int32_t>(fused_partials_per_row(t->D));
+    p.T = T;
+    p.K = t->desc.K;
+    p.shared_noise = t->independent ? 0 : 1;
+    p.node_id_base = static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap);
+    p.keys = make_philox_keys(t->desc.seed);
+    p.mix_shared = t->mix_shared;
+    p.mix_innov = t->mix_innov;
+    const cudaError_t e = launch_rollout_fused(p, static_cast<int32_t>(off), as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "whole-tree rollout kernel");
+    // host mirror of the finished tree
+    int32_t w = 1;
+    for (int i = 0; i < T; ++i) {
+        const int fan = ((p.split_bits >> i) & 1ull) ? t->desc.K : 1;
+        t->lv.fanout[i] = fan;
+        w *= fan;
+        t->lv.width[i + 1] = w;
+        t->lv.offset[i + 2] = p.off[i + 2];
+    }
+    t->pending.logp_out = nullptr;
+    t->depth = T;
     return BGRPO_OK;
 }
 

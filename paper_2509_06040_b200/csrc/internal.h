@@ -19,6 +19,22 @@ constexpr int kStepVec = 8;
 constexpr int kStepChunkVec = kStepThreads * kStepVec;   // 512 float4 = 8 KiB per operand tile
 constexpr int kStepWarps = kStepThreads / 32;            // log-prob partials per (row, chunk)
 constexpr int kStepCtasPerSm = 8;
+// Whole-tree rollout kernel: 128-thread CTAs, 2 float4 per thread (measured on B200 against 64/256 threads and 1/2/4
+// float4: within 6 % of one another), one log-prob partial per node row and warp; at most kFusedMaxSplits split steps
+// (one register-resident parent mean per split level on the depth-first walk).
+constexpr int kFusedThreads = 128;
+constexpr int kFusedVec = 2;
+constexpr int kFusedChunkVec = kFusedThreads * kFusedVec;   // float4 of a row per CTA
+constexpr int kFusedMaxSplits = 6;
+// log-prob partials of the whole-tree kernel per node row: one float per warp of every CTA that covers the row
+inline int64_t fused_partials_per_row(int64_t D) { return ((D / 4 + kFusedChunkVec - 1) / kFusedChunkVec) * (kFusedThreads / 32); }
+// floats of log-prob partials reserved per node row: the larger of the two rollout kernels' layouts
+inline int64_t partials_per_row(int64_t D) {
+    const int64_t D4 = D / 4;
+    const int64_t step = ((D4 + kStepChunkVec - 1) / kStepChunkVec) * kStepWarps;
+    const int64_t fused = fused_partials_per_row(D);
+    return step > fused ? step : fused;
+}
 constexpr int kScratchHeader = 256;    // bytes reserved at the start of scratch for the status word
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u;   // Philox4x32 multipliers and Weyl key increments (Salmon et al., SC'11)
@@ -129,6 +145,24 @@ cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s);
 
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s);
 cudaError_t launch_philox_normals(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, float* out, int64_t n, cudaStream_t s);
+
+// ---- whole-tree rollout (tree_fused.cu) -------------------------------------------------------------------------
+struct FusedLaunch {
+    float* latents;
+    const float* mu;           // [n_trees][D]
+    float* logp;
+    int32_t* table;
+    float* partialsf;          // [rows][per_row]: one float per warp of the CTAs that cover a row
+    int64_t D;
+    int32_t n_trees, nodes_cap, nchunks, per_row, T, K, shared_noise;   // nchunks: CTAs per tree
+    uint32_t node_id_base;
+    uint64_t split_bits;       // bit i: step i forks every node into K children
+    PhiloxKeys keys;
+    float mix_shared, mix_innov;
+    int32_t off[BGRPO_MAX_T + 2];                      // first local index of every depth
+    float ca[BGRPO_MAX_T], cb[BGRPO_MAX_T], g[BGRPO_MAX_T], inv_2g2[BGRPO_MAX_T], logp_const[BGRPO_MAX_T];
+};
+cudaError_t launch_rollout_fused(const FusedLaunch& p, int32_t nodes, cudaStream_t s);
 
 // ---- tree reductions (tree_reduce.cu) -------------------------------------------------------------------------
 struct FuseLaunch {

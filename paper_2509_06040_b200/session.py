@@ -21,8 +21,11 @@ class TreeSession:
     [velocity, tree_step]; rewards(); fuse_advantage(); prune().
     """
 
-    def __init__(self, w, n_trees: Optional[int] = None, tree_id_base: int = 0, device="cuda:0", nodes_cap=None):
+    def __init__(self, w, n_trees: Optional[int] = None, tree_id_base: int = 0, device="cuda:0", nodes_cap=None,
+                 fused_rollout: bool = False):
         self.w = w
+        # one launch for all T steps (closed-form velocity only) instead of one tree_step per depth
+        self.fused_rollout = fused_rollout and w.velocity == "linear"
         self.n_trees = w.n_trees if n_trees is None else n_trees
         self.device = torch.device(device)
         self.nodes_cap = w.nodes if nodes_cap is None else nodes_cap
@@ -89,6 +92,9 @@ class TreeSession:
 
     def rollout(self, seed=None):
         self.init(seed)
+        if self.fused_rollout:
+            B.tree_rollout_fused(self.tree, [1 if i in self.w.splits else 0 for i in range(self.w.T)])
+            return
         for i in range(self.w.T):
             self.step(i)
 
@@ -124,7 +130,10 @@ class TreeSession:
 
     def kernel_launches_per_pass(self) -> int:
         w = self.w
-        n = 1 + w.T * (2 if w.velocity == "mlp" else 1) + 1       # root + (mlp +) step per depth + log-prob flush
+        if self.fused_rollout:
+            n = 1 + 2                                              # root + whole-tree rollout + its log-prob sums
+        else:
+            n = 1 + w.T * (2 if w.velocity == "mlp" else 1) + 1   # root + (mlp +) step per depth + log-prob flush
         n += 1 if w.reward in ("neg_mse_mu", "neg_mse_target", "normal_plus_cos") else 0
         n += 2                                                     # fuse+advantage, prune
         return n

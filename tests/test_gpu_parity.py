@@ -475,3 +475,91 @@ def test_grpo_objective_matches_oracle(B):
             assert abs(J[t].item() - Jr) <= 1e-6 * max(1.0, abs(Jr))
             assert np.abs(terms[t].cpu().numpy() - tr).max() <= 1e-6 * max(1.0, np.abs(tr).max())
     assert J[1].item() == 0.0
+
+
+# ---------------------------------------------------------------------------------------------- whole-tree rollout in one launch
+@pytest.mark.parametrize("tokens,channels,n_trees,T,K,splits,s,sigma", [
+    (16, 4, 1, 4, 2, (0, 2), math.inf, 0.3),            # toy shape
+    (700, 12, 2, 6, 2, (0, 2, 3), math.inf, 0.3),       # several chunks and a ragged tail (D/4 = 2100), consecutive splits
+    (33, 20, 3, 5, 3, (1, 3), 2.0, 0.5),                # K = 3 with shared noise (finite s)
+    (64, 16, 1, 7, 4, (6,), 1.0, 0.3),                  # K = 4, split at the last step
+    (40, 8, 2, 6, 2, (0, 1, 2, 3, 4, 5), math.inf, 0.3),  # six splits: the deepest walk the kernel supports
+    (24, 4, 1, 5, 1, (), math.inf, 0.3),                # no split at all
+])
+def test_fused_rollout_matches_oracle_and_stepwise(B, tokens, channels, n_trees, T, K, splits, s, sigma):
+    w = Workload(name="fused", n_trees=n_trees, tokens=tokens, channels=channels, T=T, K=K, splits=splits, sigma=sigma,
+                 velocity="linear", reward="neg_mse_mu", branch_corr_s=s)
+    inp = make_inputs(w)
+    topo, lat, logp = oracle_rollout(w, inp, n_trees)
+    fused = _session(w, fused_rollout=True)
+    fused.upload_inputs(inp)
+    fused.rollout()
+    step = _session(w)
+    step.upload_inputs(inp)
+    step.rollout()
+    torch.cuda.synchronize()
+    B.tree_sync_status(fused.tree)
+    assert_table(fused, topo, n_trees)
+    assert B.tree_stats(fused.tree) == B.tree_stats(step.tree)
+    got = fused.latents.cpu().numpy()[:, :topo.nodes]
+    assert np.abs(got - lat).max() <= LATENT_TOL
+    assert np.abs(fused.logp.cpu().numpy()[:, :topo.nodes] - logp).max() <= LOGP_TOL
+    # the same draws and the same float32 expressions as the level-by-level kernel: identical latents
+    assert np.array_equal(got, step.latents.cpu().numpy()[:, :topo.nodes])
+    assert np.array_equal(fused.node_table.cpu().numpy(), step.node_table.cpu().numpy())
+    # the reductions run on a tree grown either way
+    fused.rewards(); fused.fuse_advantage(); fused.prune()
+    step.rewards(); step.fuse_advantage(); step.prune()
+    torch.cuda.synchronize()
+    assert np.array_equal(fused.mask.cpu().numpy(), step.mask.cpu().numpy())
+    assert np.allclose(fused.adv.cpu().numpy(), step.adv.cpu().numpy(), rtol=1e-4, atol=1e-4)
+
+
+def test_fused_rollout_hybrid_schedule_and_errors(B):
+    """ODE steps of the hybrid schedule (sigma = 0: child = mean, log-prob 0) and the call's error paths."""
+    w = Workload(name="fused_mix", n_trees=1, tokens=50, channels=8, T=6, K=2, splits=(1, 3), sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    inp = make_inputs(w)
+    flags = [1 if i in w.splits else 0 for i in range(w.T)]
+    sde_flags = [0, 1, 0, 1, 1, 0]
+    a = _session(w)
+    a.upload_inputs(inp)
+    a.init()
+    B.tree_set_sde_steps(a.tree, sde_flags)
+    B.tree_rollout_fused(a.tree, flags)
+    b = _session(w)
+    b.upload_inputs(inp)
+    b.init()
+    B.tree_set_sde_steps(b.tree, sde_flags)
+    for i in range(w.T):
+        B.tree_step(b.tree, flags[i])
+    torch.cuda.synchronize()
+    assert np.array_equal(a.latents.cpu().numpy(), b.latents.cpu().numpy())
+    assert np.abs(a.logp.cpu().numpy() - b.logp.cpu().numpy()).max() <= LOGP_TOL
+    assert np.all(a.logp.cpu().numpy()[0, 1:2] == 0.0)                 # step 0 is an ODE step
+    with pytest.raises(B.BgrpoError) as e:                             # the tree is complete
+        B.tree_rollout_fused(a.tree, flags)
+    assert e.value.status == B.ERR_STATE
+    c = _session(w)
+    c.upload_inputs(inp)
+    c.init()
+    B.tree_set_sde_steps(c.tree, [0, 0, 1, 1, 1, 1])
+    with pytest.raises(B.BgrpoError) as e:                             # split on an ODE step
+        B.tree_rollout_fused(c.tree, flags)
+    assert e.value.status == B.ERR_INVALID_ARG
+    w7 = Workload(name="fused7", n_trees=1, tokens=8, channels=4, T=7, K=2, splits=tuple(range(7)), sigma=0.3,
+                  velocity="linear", reward="neg_mse_mu")
+    d = _session(w7)
+    d.upload_inputs(make_inputs(w7))
+    d.init()
+    with pytest.raises(B.BgrpoError) as e:                             # seven split steps
+        B.tree_rollout_fused(d.tree, [1] * 7)
+    assert e.value.status == B.ERR_UNSUPPORTED
+    wm = Workload(name="fused_mlp", n_trees=1, tokens=8, channels=64, T=2, K=2, splits=(0,), sigma=0.3,
+                  velocity="mlp", reward="mixture", hidden=128)
+    m = _session(wm)
+    m.upload_inputs(make_inputs(wm))
+    m.init()
+    with pytest.raises(B.BgrpoError) as e:                             # no bound closed-form velocity
+        B.tree_rollout_fused(m.tree, [1, 0])
+    assert e.value.status == B.ERR_STATE
