@@ -65,6 +65,24 @@ def fuse_rewards(topo: Topology, leaf_rewards: Sequence[float], edge_logp: Optio
     return rbar
 
 
+def fusion_ess(topo: Topology, edge_logp: Optional[np.ndarray] = None, beta: float = 0.0,
+               logp_scale: float = 1.0) -> np.ndarray:
+    """Effective sample size of the fusion weights of every node (appendix "Reward Fusion: Unbiasedness and
+    Variance Reduction"): ESS(n) = (sum_l w_l)^2 / sum_l w_l^2 over the descendant leaves of n, with the
+    weights of Eq. 3, w_l proportional to exp(beta * s_l).  By direct enumeration, like fuse_rewards.
+    beta = 0 gives |L(n)|; one dominant leaf gives 1."""
+    ess = np.zeros(topo.nodes, dtype=np.float64)
+    for n in range(topo.nodes):
+        leaves = topo.descendant_leaves(n)
+        if beta == 0.0 or edge_logp is None:
+            a = np.zeros(len(leaves))
+        else:
+            a = np.array([beta * logp_scale * path_logp(topo, edge_logp, n, l) for l in leaves])
+        w = np.exp(a - a.max())
+        ess[n] = float(w.sum() ** 2 / (w ** 2).sum())
+    return ess
+
+
 def depth_advantages(topo: Topology, rbar: np.ndarray, eps: float = 1e-6, clip: float = 0.0) -> np.ndarray:
     """A_d(n) = (rbar(n) - mu_d) / (sigma_d + eps) over the nodes of each depth d >= 1 (Eq. 4);
     the edge into n carries A(n); optional clipping to [-clip, clip] when clip > 0."""

@@ -74,7 +74,10 @@ __device__ __forceinline__ void emit_child(const FusedLaunch& p, const Ctx& cx, 
 
 // Walks the subtree below local node j of depth i, whose latent pieces are in z.  S counts the splits on the path so
 // far: each split level keeps its parent's mean in registers while the children's subtrees are walked one by one.
-template <int S>
+// MAXS bounds the number of split levels the instantiation walks, SHARED says whether split steps mix in a per-parent
+// xi_0 (finite s): the common case (few splits, independent children) then carries neither the deeper levels' code nor
+// registers for xi_0.
+template <int S, int MAXS, bool SHARED>
 __device__ __forceinline__ void walk(const FusedLaunch& p, const Ctx& cx, int i, int j, int split_step, int branch_id,
                                      float4 (&z)[kFusedVec]) {
     const float4 zero[kFusedVec] = {};
@@ -90,8 +93,8 @@ __device__ __forceinline__ void walk(const FusedLaunch& p, const Ctx& cx, int i,
             emit_child(p, cx, i, parent_local, p.off[i + 1] + j, split_step, branch_id, g, m, zero, false, z);
             continue;
         }
-        if constexpr (S < kFusedMaxSplits) {
-            const bool shared = p.shared_noise != 0 && g != 0.0f;
+        if constexpr (S < MAXS) {
+            const bool shared = SHARED && g != 0.0f;
             float4 xi0[kFusedVec] = {};
             if (shared) {
 #pragma unroll
@@ -103,13 +106,14 @@ __device__ __forceinline__ void walk(const FusedLaunch& p, const Ctx& cx, int i,
                 float4 c[kFusedVec];
                 const int child = j * p.K + b;
                 emit_child(p, cx, i, parent_local, p.off[i + 1] + child, i, b, g, m, xi0, shared, c);
-                walk<S + 1>(p, cx, i + 1, child, i, b, c);
+                walk<S + 1, MAXS, SHARED>(p, cx, i + 1, child, i, b, c);
             }
         }
         return;
     }
 }
 
+template <int MAXS, bool SHARED>
 __global__ void __launch_bounds__(kFusedThreads)
 rollout_fused_kernel(const __grid_constant__ FusedLaunch p) {
     Ctx cx;
@@ -135,7 +139,7 @@ rollout_fused_kernel(const __grid_constant__ FusedLaunch p) {
             z[k] = __ldcs(cx.tree_base + cx.e[k]);          // root latent (row 0 of the tree)
         }
     }
-    walk<0>(p, cx, 0, 0, -1, 0, z);
+    walk<0, MAXS, SHARED>(p, cx, 0, 0, -1, 0, z);
 }
 
 // Completes the log-probs of every non-root node of every tree from the fused kernel's partial sums: one warp per node
@@ -171,7 +175,16 @@ finalize_tree_kernel(const __grid_constant__ FusedLaunch p, int32_t nodes) {
 cudaError_t launch_rollout_fused(const FusedLaunch& p, int32_t nodes, cudaStream_t s) {
     const int64_t items = static_cast<int64_t>(p.n_trees) * p.nchunks;
     if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    rollout_fused_kernel<<<static_cast<unsigned int>(items), kFusedThreads, 0, s>>>(p);
+    const unsigned int grid = static_cast<unsigned int>(items);
+    const int n_splits = __builtin_popcountll(p.split_bits);
+    if (n_splits > kFusedMaxSplits) return cudaErrorInvalidValue;
+    if (p.shared_noise) {
+        if (n_splits <= 3) rollout_fused_kernel<3, true><<<grid, kFusedThreads, 0, s>>>(p);
+        else rollout_fused_kernel<kFusedMaxSplits, true><<<grid, kFusedThreads, 0, s>>>(p);
+    } else {
+        if (n_splits <= 3) rollout_fused_kernel<3, false><<<grid, kFusedThreads, 0, s>>>(p);
+        else rollout_fused_kernel<kFusedMaxSplits, false><<<grid, kFusedThreads, 0, s>>>(p);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || nodes < 2) return e;
     const int64_t warps = static_cast<int64_t>(p.n_trees) * (nodes - 1);

@@ -239,3 +239,39 @@ def test_mix_schedule():
     m = credit.gradient_mask(topo, rbar, credit.WIDTH_NONE, 0, (), False, sde_steps=[0, 3, 5])
     for n in range(1, topo.nodes):
         assert m[n] == int(topo.depth[n] - 1 in (0, 3, 5))
+
+
+# ---------------------------------------------------------------------------------------------- ESS of the fusion weights
+def test_fusion_ess_special_cases_and_bounds():
+    """Appendix "Reward Fusion": ESS = (sum w)^2 / sum w^2.  beta = 0 -> the number of descendant leaves; equal edge
+    log-probs -> the same for any beta; a two-leaf node with path probabilities (p, 1-p) at beta = 1 -> 1/(p^2+(1-p)^2);
+    one overwhelming leaf -> 1; always 1 <= ESS <= |L(n)|."""
+    topo = tree.build_topology(5, 3, (0, 2, 3))
+    n_leaves = np.array([len(topo.descendant_leaves(n)) for n in range(topo.nodes)], dtype=np.float64)
+    rng = np.random.default_rng(5)
+    logp = rng.normal(-1.0, 0.7, size=topo.nodes)
+    assert np.allclose(credit.fusion_ess(topo, logp, 0.0), n_leaves)
+    assert np.allclose(credit.fusion_ess(topo, np.full(topo.nodes, -0.3), 2.5), n_leaves)
+    for beta in (0.5, 1.0, 4.0):
+        ess = credit.fusion_ess(topo, logp, beta)
+        assert np.all(ess >= 1.0 - 1e-12) and np.all(ess <= n_leaves + 1e-9)
+        assert np.allclose(ess[topo.offset[topo.T]:], 1.0)               # a leaf is its own only descendant
+    # two leaves under one parent, probabilities p and 1 - p
+    t2 = tree.build_topology(1, 2, (0,))
+    p = 0.8
+    lp = np.array([0.0, math.log(p), math.log(1 - p)])
+    assert credit.fusion_ess(t2, lp, 1.0)[0] == pytest.approx(1.0 / (p * p + (1 - p) * (1 - p)), rel=1e-12)
+    # textbook form on explicit normalised weights
+    t3 = tree.build_topology(2, 2, (0, 1))
+    lp3 = rng.normal(size=t3.nodes)
+    s = np.array([credit.path_logp(t3, lp3, 0, l) for l in t3.leaf_ids()])
+    w = special.softmax(1.3 * s)
+    assert credit.fusion_ess(t3, lp3, 1.3)[0] == pytest.approx(1.0 / np.sum(w ** 2), rel=1e-12)
+    # one leaf overwhelmingly likely
+    lp_dom = np.full(t3.nodes, -50.0)
+    leaf = t3.leaf_ids()[2]
+    m = leaf
+    while m > 0:
+        lp_dom[m] = 0.0
+        m = int(t3.parent[m])
+    assert credit.fusion_ess(t3, lp_dom, 1.0)[0] == pytest.approx(1.0, abs=1e-12)
