@@ -184,6 +184,13 @@ bgrpo_status bgrpo_leaf_reward_cos(bgrpo_tree* tree, const float* target_dev, fl
 bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* tree, const float* leaf_rewards_dev, float beta, float logp_scale,
                                        float eps, float adv_clip_max, void* stream);
 
+/* Effective sample size of the fusion weights of every node (appendix "Reward Fusion: Unbiasedness and Variance
+ * Reduction"): ESS(n) = (sum_l w_l)^2 / sum_l w_l^2 over the descendant leaves l of n, with the weights of Eq. 3,
+ * w_l = exp(beta * logp_scale * s_l).  A diagnostic of how far path-probability weighting concentrates on a few leaves:
+ * beta = 0 gives the number of descendant leaves, one dominant leaf gives 1.  Reads buffers.logp of a complete tree.
+ * ess_out_dev: device [n_trees][nodes_cap] float32. */
+bgrpo_status bgrpo_tree_fusion_ess(bgrpo_tree* tree, float beta, float logp_scale, float* ess_out_dev, void* stream);
+
 /* tree_prune: gradient mask per node-step; reads buffers.rbar, writes buffers.mask only ("pruning ... affects
  * backpropagation but not forward rollouts or reward evaluation").  mask(n) = keep_width(n) AND step(depth(n)-1) not in
  * pruned_steps AND n is not the root AND (ignore_last_step == 0 OR depth(n) < T).  Width ranking compares the float32

@@ -71,6 +71,7 @@ _SIGNATURES = {
     "bgrpo_leaf_reward_mse": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "bgrpo_leaf_reward_cos": (C.c_int, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_fuse_advantage": (C.c_int, [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_float, C.c_void_p]),
+    "bgrpo_tree_fusion_ess": (C.c_int, [C.c_void_p, C.c_float, C.c_float, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_prune": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, _i32p, C.c_int32, C.c_int32, C.c_void_p]),
     "bgrpo_tree_grpo_objective": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_set_sde_steps": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -203,6 +204,10 @@ def leaf_reward_cos(tree: Tree, target, scale: float, r_inout, stream=None):
 def tree_fuse_advantage(tree: Tree, leaf_rewards, beta=0.0, logp_scale=1.0, eps=1e-6, adv_clip_max=0.0, stream=None):
     _check(lib.bgrpo_tree_fuse_advantage(tree.handle, _ptr(leaf_rewards), beta, logp_scale, eps, adv_clip_max,
                                          _stream(stream)), "bgrpo_tree_fuse_advantage")
+
+
+def tree_fusion_ess(tree: Tree, beta: float, logp_scale: float, ess_out, stream=None):
+    _check(lib.bgrpo_tree_fusion_ess(tree.handle, beta, logp_scale, _ptr(ess_out), _stream(stream)), "bgrpo_tree_fusion_ess")
 
 
 def tree_prune(tree: Tree, width_mode: int, k_or_b: int, pruned_steps: Sequence[int] = (), ignore_last_step=False,

@@ -49,6 +49,7 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     size_t b = kScratchHeader;
     b += ((static_cast<size_t>(rows) * sizeof(unsigned int) + 255) / 256) * 256;
     b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
+    b += static_cast<size_t>(rows) * 2 * sizeof(double);
     b += static_cast<size_t>(rows) * static_cast<size_t>(partials_per_row(D)) * sizeof(float);
     return b;
 }
@@ -189,7 +190,8 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     t->status = reinterpret_cast<int32_t*>(sc);
     t->counters = reinterpret_cast<unsigned int*>(sc + kScratchHeader);
     t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
-    t->partialsf = reinterpret_cast<float*>(t->partials + rows * static_cast<size_t>(t->nchunks) * 3);
+    t->node_scratch = t->partials + rows * static_cast<size_t>(t->nchunks) * 3;
+    t->partialsf = reinterpret_cast<float*>(t->node_scratch + rows * 2);
     t->pending.logp_out = nullptr;
     fill_coefficients(t);
     st = bgrpo_tree_reset(t, desc->seed, stream);
@@ -425,6 +427,7 @@ bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* t, const float* leaf_rewards_
     p.rbar = t->buf.rbar;
     p.adv = t->buf.adv;
     p.status = t->status;
+    p.node_scratch = t->node_scratch;
     p.lv = t->lv;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
@@ -433,9 +436,27 @@ bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* t, const float* leaf_rewards_
     p.beta_scaled = static_cast<double>(beta) * static_cast<double>(logp_scale);
     p.eps = eps;
     p.clip = adv_clip_max;
-    if (static_cast<size_t>(p.nodes) * 16 > 200 * 1024) return fail(BGRPO_ERR_UNSUPPORTED, "tree too large for one CTA's shared memory");
     cudaError_t e = launch_fuse_advantage(p, as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "fuse kernel");
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_fusion_ess(bgrpo_tree* t, float beta, float logp_scale, float* ess_out_dev, void* stream) {
+    if (!t || !ess_out_dev) return fail(BGRPO_ERR_INVALID_ARG, "tree or output is NULL");
+    if (!tree_complete(t)) return fail(BGRPO_ERR_STATE, "tree is not complete");
+    if (!std::isfinite(beta) || !std::isfinite(logp_scale)) return fail(BGRPO_ERR_INVALID_ARG, "beta and logp_scale must be finite");
+    EssLaunch p;
+    p.logp = t->buf.logp;
+    p.ess = ess_out_dev;
+    p.node_scratch = t->node_scratch;
+    p.lv = t->lv;
+    p.n_trees = t->desc.n_trees;
+    p.nodes_cap = t->desc.nodes_cap;
+    p.T = t->desc.T;
+    p.nodes = t->lv.offset[t->desc.T + 1];
+    p.beta_scaled = static_cast<double>(beta) * static_cast<double>(logp_scale);
+    const cudaError_t e = launch_fusion_ess(p, as_stream(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "fusion ESS kernel");
     return BGRPO_OK;
 }
 

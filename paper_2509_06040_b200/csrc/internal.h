@@ -106,7 +106,9 @@ struct bgrpo_tree {
     int32_t* status;
     unsigned int* counters;              // one ticket counter per (tree, node row)
     double* partials;                    // [n_trees*nodes_cap][nchunks][3]   (reward reductions)
-    float* partialsf;                    // [n_trees*nodes_cap][nchunks_step][kStepWarps] (log-prob sums of the step kernel)
+    double* node_scratch;                // [n_trees][2][nodes_cap]: per-node state of the tree reductions when a tree
+                                         // is too large for one CTA's shared memory
+    float* partialsf;                    // [n_trees*nodes_cap][partials_per_row] (log-prob sums of the rollout kernels)
     bgrpo::FinalizeDesc pending;         // level whose log-probs still have to be summed
 };
 
@@ -165,11 +167,19 @@ struct FusedLaunch {
 cudaError_t launch_rollout_fused(const FusedLaunch& p, int32_t nodes, cudaStream_t s);
 
 // ---- tree reductions (tree_reduce.cu) -------------------------------------------------------------------------
+constexpr size_t kTreeSmemLimit = 200 * 1024;   // per-node doubles beyond this live in node_scratch instead of shared memory
 struct FuseLaunch {
     const float* leaf_r; const float* logp; float* rbar; float* adv; int32_t* status;
+    double* node_scratch;      // [n_trees][2][nodes_cap], used when 16 bytes per node exceed kTreeSmemLimit
     LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes; double beta_scaled; float eps, clip;
 };
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s);
+
+struct EssLaunch {
+    const float* logp; float* ess; double* node_scratch;
+    LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes; double beta_scaled;
+};
+cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s);
 
 struct PruneLaunch {
     const float* rbar; const int32_t* table; uint8_t* mask;

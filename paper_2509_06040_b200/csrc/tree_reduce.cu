@@ -1,6 +1,8 @@
 // Tree reductions: reward fusion (Eq. 3) + depth-wise normalisation (Eq. 4) in one kernel, and the width / depth
 // pruning masks ("Pruning Strategies") in another.  A tree has at most a few thousand nodes, so one CTA owns one
 // tree, keeps the per-node state in shared memory as doubles and walks the levels; the kernels are latency-bound.
+// A tree whose per-node state does not fit in shared memory (more than 12 800 nodes: K = 4 with seven splits, say)
+// keeps it in the caller's scratch instead; the code is the same, only the pointer differs.
 //
 // Fusion uses the bottom-up form of Eq. 3.  With a_c = beta*logp(c) the softmax weight of leaf l under node n
 // factorises along the path, so  S_n = sum_c e^{a_c} S_c,  R_n = sum_c e^{a_c} R_c,  rbar(n) = R_n / S_n  with
@@ -22,9 +24,10 @@ __device__ __forceinline__ double warp_sum_d(double x) {
 __global__ void __launch_bounds__(kTreeThreads)
 fuse_advantage_kernel(const FuseLaunch p) {
     extern __shared__ double sm[];
-    double* rb = sm;                 // rbar per node
-    double* ls = sm + p.nodes;       // log S per node
     const int tree = blockIdx.x;
+    const bool in_smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double) <= kTreeSmemLimit;
+    double* rb = in_smem ? sm : p.node_scratch + static_cast<int64_t>(tree) * 2 * p.nodes_cap;   // rbar per node
+    double* ls = rb + (in_smem ? p.nodes : p.nodes_cap);                                          // log S per node
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     const int T = p.T;
     const int leaves = p.lv.width[T];
@@ -86,6 +89,58 @@ fuse_advantage_kernel(const FuseLaunch p) {
             p.adv[row0 + off + j] = static_cast<float>(A);
             p.rbar[row0 + off + j] = static_cast<float>(rb[off + j]);
         }
+    }
+}
+
+// Effective sample size of the fusion weights (appendix "Reward Fusion"): ESS(n) = (sum_l w_l)^2 / sum_l w_l^2 over the
+// descendant leaves of n, w_l = exp(beta s_l).  Both sums factorise along the paths like S above:
+//   log S_n = logsumexp_c(a_c + log S_c),   log Q_n = logsumexp_c(2 a_c + log Q_c),   ESS = exp(2 log S - log Q).
+__global__ void __launch_bounds__(kTreeThreads)
+fusion_ess_kernel(const EssLaunch p) {
+    extern __shared__ double sm[];
+    const int tree = blockIdx.x;
+    const bool in_smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double) <= kTreeSmemLimit;
+    double* ls = in_smem ? sm : p.node_scratch + static_cast<int64_t>(tree) * 2 * p.nodes_cap;
+    double* lq = ls + (in_smem ? p.nodes : p.nodes_cap);
+    const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
+    const int T = p.T;
+    for (int l = threadIdx.x; l < p.lv.width[T]; l += kTreeThreads) {
+        ls[p.lv.offset[T] + l] = 0.0;
+        lq[p.lv.offset[T] + l] = 0.0;
+        p.ess[row0 + p.lv.offset[T] + l] = 1.0f;
+    }
+    __syncthreads();
+    for (int d = T - 1; d >= 0; --d) {
+        const int fan = p.lv.fanout[d];
+        const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
+        for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads) {
+            const int c0 = offc + j * fan;
+            double a1[BGRPO_MAX_K], a2[BGRPO_MAX_K];
+            double m1 = -INFINITY, m2 = -INFINITY;
+#pragma unroll
+            for (int b = 0; b < BGRPO_MAX_K; ++b) {
+                if (b < fan) {
+                    const double a = p.beta_scaled * static_cast<double>(p.logp[row0 + c0 + b]);
+                    a1[b] = a + ls[c0 + b];
+                    a2[b] = 2.0 * a + lq[c0 + b];
+                    m1 = fmax(m1, a1[b]);
+                    m2 = fmax(m2, a2[b]);
+                }
+            }
+            double S = 0.0, Q = 0.0;
+#pragma unroll
+            for (int b = 0; b < BGRPO_MAX_K; ++b) {
+                if (b < fan) {
+                    S += exp(a1[b] - m1);
+                    Q += exp(a2[b] - m2);
+                }
+            }
+            const double lS = m1 + log(S), lQ = m2 + log(Q);
+            ls[off + j] = lS;
+            lq[off + j] = lQ;
+            p.ess[row0 + off + j] = static_cast<float>(exp(2.0 * lS - lQ));
+        }
+        __syncthreads();
     }
 }
 
@@ -196,8 +251,20 @@ cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s) {
+    size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);
+    if (smem > kTreeSmemLimit) smem = 0;          // per-node state in the caller's scratch
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(fusion_ess_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    fusion_ess_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
-    const size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);
+    size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);
+    if (smem > kTreeSmemLimit) smem = 0;          // per-node state in the caller's scratch
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(fuse_advantage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;

@@ -563,3 +563,70 @@ def test_fused_rollout_hybrid_schedule_and_errors(B):
     with pytest.raises(B.BgrpoError) as e:                             # no bound closed-form velocity
         B.tree_rollout_fused(m.tree, [1, 0])
     assert e.value.status == B.ERR_STATE
+
+
+# ---------------------------------------------------------------------------------------------- path-weighted fusion at scale, ESS, large trees
+@pytest.mark.parametrize("T,K,splits", [(6, 3, (0, 1, 3, 4)), (5, 4, (0, 1, 2, 4)), (20, 3, (0, 3, 6, 9))])
+def test_path_weighted_fusion_and_ess_on_wide_trees(B, T, K, splits):
+    """K = 3 / 4 trees with 81 / 256 leaves (the paper's scaling study), beta = 1 (the ablation's path-probability
+    weighting) on joint log-densities (logp_scale = D): fused values, advantages and the effective sample size of the
+    weights against the oracle's enumeration, teacher-forced with the same float32 log-probs and rewards."""
+    w, s, topo = _grown_session(B, T, K, splits, n_trees=2, D_tokens=8)
+    assert topo.leaves in (81, 256)
+    rng = np.random.default_rng(K * 100 + T)
+    r = rng.standard_normal((2, topo.leaves)).astype(np.float32)
+    lp = (-0.9 + 0.15 * rng.standard_normal((2, topo.nodes))).astype(np.float32)      # per-element means: close together
+    lp[:, 0] = 0
+    s.logp.copy_(torch.from_numpy(lp))
+    r_dev = torch.from_numpy(r).cuda()
+    ess = torch.empty_like(s.logp)
+    for beta, scale in ((1.0, float(w.D)), (0.0, 1.0), (2.5, 1.0)):
+        B.tree_fuse_advantage(s.tree, r_dev, beta, scale, 1e-6, 0.0)
+        B.tree_fusion_ess(s.tree, beta, scale, ess)
+        torch.cuda.synchronize()
+        for t in range(2):
+            rbar = credit.fuse_rewards(topo, r[t], lp[t].astype(np.float64), beta, scale)
+            adv = credit.depth_advantages(topo, rbar, 1e-6)
+            ref_ess = credit.fusion_ess(topo, lp[t].astype(np.float64), beta, scale)
+            assert np.abs(s.rbar.cpu().numpy()[t] - rbar).max() <= 1e-6 * max(1.0, np.abs(rbar).max())
+            assert adv_close(s.adv.cpu().numpy()[t], adv), (beta, scale, t)
+            got_ess = ess.cpu().numpy()[t, :topo.nodes]
+            assert np.all(np.abs(got_ess - ref_ess) <= 1e-5 * ref_ess), (beta, scale, t)
+            if beta == 0.0:
+                assert got_ess[0] == topo.leaves
+    B.tree_sync_status(s.tree)
+
+
+def test_reductions_on_a_tree_larger_than_shared_memory(B):
+    """K = 4 with seven splits: 21 845 nodes, more than one CTA's shared memory holds as doubles; the reduction kernels
+    keep their per-node state in the caller's scratch instead.  Fusion, advantages, ESS and masks against the oracle."""
+    T, K, splits = 7, 4, tuple(range(7))
+    w = Workload(name="huge", n_trees=2, tokens=1, channels=4, T=T, K=K, splits=splits, sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    s = _session(w)
+    s.upload_inputs(make_inputs(w))
+    s.rollout()
+    topo = otree.build_topology(T, K, splits)
+    assert topo.nodes == 21845 and topo.nodes * 16 > 200 * 1024
+    rng = np.random.default_rng(77)
+    r = rng.standard_normal((2, topo.leaves)).astype(np.float32)
+    lp = (-1.0 + 0.4 * rng.standard_normal((2, topo.nodes))).astype(np.float32)
+    lp[:, 0] = 0
+    s.logp.copy_(torch.from_numpy(lp))
+    r_dev = torch.from_numpy(r).cuda()
+    ess = torch.empty_like(s.logp)
+    beta = 1.0
+    B.tree_fuse_advantage(s.tree, r_dev, beta, 1.0, 1e-6, 0.0)
+    B.tree_fusion_ess(s.tree, beta, 1.0, ess)
+    B.tree_prune(s.tree, B.WIDTH_PER_SPLIT_TOPK, 2, (1, 4), False)
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    t = 1
+    rbar = credit.fuse_rewards(topo, r[t], lp[t].astype(np.float64), beta, 1.0)
+    adv = credit.depth_advantages(topo, rbar, 1e-6)
+    assert np.abs(s.rbar.cpu().numpy()[t] - rbar).max() <= 1e-6 * max(1.0, np.abs(rbar).max())
+    assert adv_close(s.adv.cpu().numpy()[t], adv)
+    ref_ess = credit.fusion_ess(topo, lp[t].astype(np.float64), beta, 1.0)
+    assert np.all(np.abs(ess.cpu().numpy()[t] - ref_ess) <= 1e-5 * ref_ess)
+    mask = credit.gradient_mask(topo, s.rbar.cpu().numpy()[t], B.WIDTH_PER_SPLIT_TOPK, 2, (1, 4), False)
+    assert np.array_equal(s.mask.cpu().numpy()[t], mask)
