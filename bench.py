@@ -304,6 +304,50 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
     return roof, roof_step, breakdown
 
 
+def fused_rollout_line(w, device, peaks, reps):
+    """The same pass with all T steps in one launch (closed-form velocity): whole-pass throughput, and the rollout
+    kernel alone against the bytes it must move (every node written once, root and target mean read once)."""
+    import torch
+    from paper_2509_06040_b200.session import TreeSession
+    from paper_2509_06040_b200 import binding as B
+    s = TreeSession(w, device=device, fused_rollout=True)
+    s.upload_inputs(make_inputs(w))
+    for k in range(2):
+        s.run_all(seed=w.seed + k)
+    torch.cuda.synchronize()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for k in range(reps):
+        s.run_all(seed=w.seed + 100 + k)
+    a1.record()
+    torch.cuda.synchronize()
+    ms = a0.elapsed_time(a1) / reps
+    flags = [1 if i in w.splits else 0 for i in range(w.T)]
+    t_k = 0.0
+    for k in range(reps):
+        s.init(seed=w.seed + 200 + k)
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record()
+        B.tree_rollout_fused(s.tree, flags)
+        b1.record()
+        torch.cuda.synchronize()
+        t_k += b0.elapsed_time(b1)
+    t_k /= reps
+    B.tree_sync_status(s.tree)
+    nbytes = w.n_trees * (w.node_steps + 2) * 4.0 * w.D
+    gbs = nbytes / (t_k * 1e-3) / 1e9
+    out = {"value": w.n_trees * w.node_steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": reps,
+           "gpu_launches_per_pass": s.kernel_launches_per_pass(),
+           "roofline": {"bound": "hbm", "kernel": "rollout_fused_kernel (+ its log-prob sums)", "achieved": gbs,
+                        "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
+                        "peak_source": peaks["_source"], "bytes_per_launch": nbytes, "ms_per_launch": t_k, "traffic": None,
+                        "note": "4 bytes per element and node-step (write only); the kernel is bound by instruction issue "
+                                "(Philox + Box-Muller), like the step kernel on this workload"}}
+    del s
+    torch.cuda.empty_cache()
+    return out
+
+
 # ------------------------------------------------------------------------------------------------ GPU arm
 def run_ours(args, w):
     import torch
@@ -429,6 +473,8 @@ def run_ours(args, w):
                           "l2": "latent pool larger than L2", "roofline": r2, "roofline_step": rs2, "kernel_ms_per_pass": bd2}
             del s2
             torch.cuda.empty_cache()
+            if w2.velocity == "linear":
+                also[name]["fused_rollout"] = fused_rollout_line(w2, f"cuda:{local}", peaks, n2)
 
     # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
     cpu = None

@@ -3,6 +3,7 @@
 #include <cstddef>
 #include <cstdint>
 #include <cuda_runtime.h>
+#include <utility>
 
 #include "../../include/bgrpo.h"
 
@@ -113,6 +114,29 @@ struct bgrpo_tree {
 };
 
 namespace bgrpo {
+
+// Programmatic dependent launch: a kernel launched with launch_overlapped() may be scheduled while the kernel before it
+// on the stream is still draining, so the gap between two dependent launches shrinks to the set-up the new kernel can do
+// on its own.  Such a kernel calls pdl_wait() before it touches anything an earlier kernel wrote or still reads, and
+// pdl_release() as early as it likes to let its own successor in.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... Params, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 
 // ---- streaming kernels (tree_step.cu) -------------------------------------------------------------------------
 struct StepLaunch {

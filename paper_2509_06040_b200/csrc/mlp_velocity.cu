@@ -280,6 +280,10 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // Barriers and tensor memory are set up: the next kernel on the stream may be scheduled, and this one waits here for
+    // the kernels before it (they wrote the latents and the packed weights, and may still be reading the output buffer).
+    pdl_release();
+    pdl_wait();
     const uint32_t tmem = sm.tmem_base;
     const int n_my_tiles = (p.n_tiles > static_cast<int>(blockIdx.x)) ? (p.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
     const int NC = p.n_chunks;
@@ -585,8 +589,7 @@ cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_of
     a.n_tiles = static_cast<int32_t>(tiles);
     a.status = status;
     const int grid = a.n_tiles < sms ? a.n_tiles : sms;
-    mlp_velocity_kernel<<<grid, kMlpThreads, sizeof(MlpSmem) + 1024, s>>>(a);
-    return cudaGetLastError();
+    return launch_overlapped(mlp_velocity_kernel, grid, kMlpThreads, sizeof(MlpSmem) + 1024, s, a);
 }
 
 }  // namespace bgrpo

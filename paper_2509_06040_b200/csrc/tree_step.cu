@@ -214,6 +214,8 @@ template <int FAN, bool SHARED, bool WRITE>
 __global__ void __launch_bounds__(kStepThreads, kStepCtasPerSm)
 step_kernel(const __grid_constant__ StepLaunch p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_release();
+    pdl_wait();           // the parents, the velocity and the pending partial sums come from earlier kernels
     // the previous level's log-probs (a handful of rows): summed by this launch
     if (p.prev.logp_out != nullptr)
         finalize_rows(p.prev, p.partialsf, p.n_trees, p.nodes_cap, p.nchunks, p.D, blockIdx.x * kStepWarps + warp, gridDim.x * kStepWarps);
@@ -342,10 +344,9 @@ __global__ void philox_normals_kernel(const __grid_constant__ PhiloxKeys keys, u
 
 template <int FAN>
 cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t s) {
-    if (!p.write_children) step_kernel<FAN, false, false><<<grid, kStepThreads, 0, s>>>(p);
-    else if (p.shared_noise) step_kernel<FAN, true, true><<<grid, kStepThreads, 0, s>>>(p);
-    else step_kernel<FAN, false, true><<<grid, kStepThreads, 0, s>>>(p);
-    return cudaGetLastError();
+    if (!p.write_children) return launch_overlapped(step_kernel<FAN, false, false>, grid, kStepThreads, 0, s, p);
+    if (p.shared_noise) return launch_overlapped(step_kernel<FAN, true, true>, grid, kStepThreads, 0, s, p);
+    return launch_overlapped(step_kernel<FAN, false, true>, grid, kStepThreads, 0, s, p);
 }
 
 }  // namespace
