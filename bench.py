@@ -42,10 +42,12 @@ NOMINAL_HBM_GBS = 8000.0
 # reported per launch is bytes-per-unit times the units of an average launch of the timed workload (traffic grows in
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
-    "step_kernel": {"workload": "video", "bytes": 75.599104e6 + 12.592896e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "d6ef704e319c"},
-    "mlp_velocity_kernel": {"workload": "8 image-shaped trees, frontier width 16", "bytes": 67.183616e6 + 15.853056e6,
-                            "units": 259200, "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "d8e9e9052c8b"},
+    "step_kernel": {"workload": "video", "bytes": 75.601408e6 + 12.221184e6, "units": 8 * 2096640,
+                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "2126f58c27b4"},
+    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.264832e6 + 214.634752e6, "units": 1036800,
+                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "f8c2d9ea6390"},
+    "rollout_fused_kernel": {"workload": "video", "bytes": 16.817664e6 + 865.891584e6, "units": 110 * 2096640,
+                             "sources": ("tree_fused.cu", "philox.cuh", "internal.h"), "source_hash": "bd5d30f37ce1"},
 }
 
 
@@ -340,7 +342,8 @@ def fused_rollout_line(w, device, peaks, reps):
            "gpu_launches_per_pass": s.kernel_launches_per_pass(),
            "roofline": {"bound": "hbm", "kernel": "rollout_fused_kernel (+ its log-prob sums)", "achieved": gbs,
                         "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
-                        "peak_source": peaks["_source"], "bytes_per_launch": nbytes, "ms_per_launch": t_k, "traffic": None,
+                        "peak_source": peaks["_source"], "bytes_per_launch": nbytes, "ms_per_launch": t_k,
+                        "traffic": ncu_traffic("rollout_fused_kernel", float(w.n_trees * w.node_steps * w.D)),
                         "note": "4 bytes per element and node-step (write only); the kernel is bound by instruction issue "
                                 "(Philox + Box-Muller), like the step kernel on this workload"}}
     del s
@@ -369,7 +372,7 @@ def run_ours(args, w):
     # weak scaling: every rank holds the workload's n_trees trees, with its own global tree indices
     base = rank * w.n_trees
     inp = make_inputs(w, tree_base=base)
-    s = TreeSession(w, tree_id_base=base, device=f"cuda:{local}")
+    s = TreeSession(w, tree_id_base=base, device=f"cuda:{local}", fused_rollout=args.fused_rollout)
     s.upload_inputs(inp)
     pool_bytes = s.latents.numel() * 4
     flush = pool_bytes <= 2 * L2_BYTES
@@ -446,7 +449,10 @@ def run_ours(args, w):
     breakdown = {}
     if rank == 0:
         peaks = load_peaks()
-        roof, roof_step, breakdown = kernel_rooflines(s, w, peaks, flush_buf, max(3, min(10, args.steps)))
+        if s.fused_rollout:
+            roof = roof_step = fused_rollout_line(w, f"cuda:{local}", peaks, max(3, min(10, args.steps)))["roofline"]
+        else:
+            roof, roof_step, breakdown = kernel_rooflines(s, w, peaks, flush_buf, max(3, min(10, args.steps)))
 
     # ---- the other image- and video-shaped workloads, briefly (rank 0, single GPU): same path, same timing method
     also = {}
@@ -494,6 +500,7 @@ def run_ours(args, w):
                        "node_steps_per_tree": w.node_steps, "model_evals_per_tree": w.model_evals,
                        "model_evals_sequential": w.leaves * w.T, "latent_pool_bytes": pool_bytes,
                        "l2": "flushed between steps (pool fits in L2)" if flush else "latent pool larger than L2",
+                       "rollout": "one launch (tree_rollout_fused)" if s.fused_rollout else "one tree_step launch per depth",
                        "parallelism": f"dp{world} over trees, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -515,6 +522,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="image", choices=list(CONFIGS))
+    ap.add_argument("--fused-rollout", action="store_true",
+                    help="closed-form-velocity workloads: all T steps in one launch (tree_rollout_fused)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="skip the brief runs of the other image/video workloads")
     args = ap.parse_args()
