@@ -51,6 +51,7 @@ size_t scratch_bytes_of(const bgrpo_tree_desc* d) {
     b += static_cast<size_t>(rows) * nchunks_of(D) * 3 * sizeof(double);
     b += static_cast<size_t>(rows) * 2 * sizeof(double);
     b += static_cast<size_t>(rows) * static_cast<size_t>(partials_per_row(D)) * sizeof(float);
+    if (d->channels == BGRPO_MLP_CHANNELS) b = ((b + 255) / 256) * 256 + kMlpTicketBytes + kMlpPartialBytes;
     return b;
 }
 
@@ -192,9 +193,20 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
     t->node_scratch = t->partials + rows * static_cast<size_t>(t->nchunks) * 3;
     t->partialsf = reinterpret_cast<float*>(t->node_scratch + rows * 2);
+    t->mlp_tickets = nullptr;
+    t->mlp_partials = nullptr;
+    if (desc->channels == BGRPO_MLP_CHANNELS) {
+        const size_t used = reinterpret_cast<char*>(t->partialsf + rows * static_cast<size_t>(partials_per_row(t->D))) - sc;
+        t->mlp_tickets = reinterpret_cast<unsigned int*>(sc + ((used + 255) / 256) * 256);
+        t->mlp_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(t->mlp_tickets) + kMlpTicketBytes);
+    }
     t->pending.logp_out = nullptr;
     fill_coefficients(t);
     st = bgrpo_tree_reset(t, desc->seed, stream);
+    if (st == BGRPO_OK && t->mlp_tickets) {      // the MLP stage's tile tickets start at zero and return to zero after every launch
+        const cudaError_t e = cudaMemsetAsync(t->mlp_tickets, 0, kMlpTicketBytes, as_stream(stream));
+        if (e != cudaSuccess) st = cuda_fail(e, "clearing the MLP tickets");
+    }
     if (st != BGRPO_OK) {
         delete t;
         return st;
@@ -214,6 +226,7 @@ bgrpo_status bgrpo_tree_reset(bgrpo_tree* t, uint64_t seed, void* stream) {
     t->lv.offset[1] = 1;
     cudaError_t e = launch_root(t, as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "root kernel");
+
     return BGRPO_OK;
 }
 
@@ -615,7 +628,7 @@ bgrpo_status bgrpo_velocity_mlp(bgrpo_tree* t, const void* packed_dev, int32_t h
     const int i = t->depth;
     cudaError_t e = launch_mlp(t->buf.latents, static_cast<int64_t>(t->desc.nodes_cap) * t->D, static_cast<int64_t>(t->lv.offset[i]) * t->D,
                                t->desc.n_trees, static_cast<int64_t>(t->lv.width[i]) * t->desc.tokens, packed_dev, hidden,
-                               v_out_dev, t->status, as_stream(stream));
+                               v_out_dev, t->mlp_partials, t->mlp_tickets, t->status, as_stream(stream));
     return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp kernel");
 }
 

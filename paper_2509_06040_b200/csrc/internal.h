@@ -110,6 +110,8 @@ struct bgrpo_tree {
     double* node_scratch;                // [n_trees][2][nodes_cap]: per-node state of the tree reductions when a tree
                                          // is too large for one CTA's shared memory
     float* partialsf;                    // [n_trees*nodes_cap][partials_per_row] (log-prob sums of the rollout kernels)
+    unsigned int* mlp_tickets;           // 64-channel trees only: scratch of the MLP stage's split over the hidden dimension
+    float* mlp_partials;
     bgrpo::FinalizeDesc pending;         // level whose log-probs still have to be summed
 };
 
@@ -218,9 +220,15 @@ struct ObjectiveLaunch {
 cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s);
 
 // ---- MLP velocity (mlp_velocity.cu) -----------------------------------------------------------------------------
+// Frontiers of fewer tiles than SMs are also cut along the hidden dimension; the partial output tiles (128 tokens x 64
+// channels, float) of at most this many CTAs and one ticket counter per tile live in the tree's scratch.
+constexpr int kMlpSplitMaxCtas = 192;
+constexpr size_t kMlpPartialBytes = static_cast<size_t>(kMlpSplitMaxCtas) * 128 * 64 * sizeof(float);
+constexpr size_t kMlpTicketBytes = 1024;      // kMlpSplitMaxCtas counters, rounded up
 size_t mlp_packed_bytes(int hidden);
 cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, void* packed, cudaStream_t s);
 cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
-                       const void* packed, int hidden, float* v_out, int32_t* status, cudaStream_t s);
+                       const void* packed, int hidden, float* v_out, float* split_partials, unsigned int* split_tickets,
+                       int32_t* status, cudaStream_t s);
 
 }  // namespace bgrpo

@@ -29,6 +29,10 @@
 // address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with
 // one copy per matrix.  No cluster multicast is used anywhere.
 //
+// Small frontiers (fewer tiles than SMs) are cut along the hidden dimension as well: S = 2, 4 or 8 CTAs share a tile, each
+// takes 1/S of the chunks and writes its partial output tile to scratch; the CTA that draws the tile's last ticket adds the
+// S partials in part order and writes v, so the result does not depend on which CTA finishes first.
+//
 // Every wait is bounded (2 s): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
 // released and bit 2 of the status word is set.
 #include "internal.h"
@@ -60,6 +64,8 @@ struct MlpSmem {
     alignas(1024) float stage[kTok * kCh];                   // float32 latents of the next tile, as they are in global memory
     unsigned long long w1_full[kW1Stages], w1_free[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
     unsigned long long stage_full, a_full[2], a_empty[2], d1_full[2], d1_empty[2], h_full[2], h_free[2], d2_full[2], d2_empty[2];
+    unsigned long long part_done, part_verdict;   // split mode: all epilogue warps have stored their partials / the ticket is drawn
+    int is_last_part;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -239,6 +245,9 @@ struct MlpArgs {
     float* v_out;
     int32_t n_chunks;         // hidden / 128
     int32_t n_tiles;
+    int32_t split;            // CTAs per tile along the hidden dimension (1: none); > 1 only with one tile per CTA group
+    float* partials;          // split > 1: [n_tiles][split][128][64] partial output tiles
+    unsigned int* tickets;    // split > 1: one counter per tile, zero before and after the launch
     int32_t* status;
 };
 
@@ -260,6 +269,8 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             mbar_init(&sm.w2_free[q], 1);
         }
         mbar_init(&sm.stage_full, 1);
+        mbar_init(&sm.part_done, kEpiWarps);
+        mbar_init(&sm.part_verdict, 1);
         for (int q = 0; q < 2; ++q) {
             mbar_init(&sm.a_full[q], 1);
             mbar_init(&sm.a_empty[q], 1);
@@ -285,8 +296,11 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
     pdl_release();
     pdl_wait();
     const uint32_t tmem = sm.tmem_base;
-    const int n_my_tiles = (p.n_tiles > static_cast<int>(blockIdx.x)) ? (p.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    const int NC = p.n_chunks;
+    const int S = p.split;
+    const int cta = static_cast<int>(blockIdx.x) / S, part = static_cast<int>(blockIdx.x) - cta * S;   // tile walker, share of the hidden dimension
+    const int n_ctas = static_cast<int>(gridDim.x) / S;
+    const int n_my_tiles = (p.n_tiles > cta) ? (p.n_tiles - 1 - cta) / n_ctas + 1 : 0;
+    const int NC = p.n_chunks / S;            // chunks this CTA adds up per tile: part * NC .. part * NC + NC - 1
     const int n_my_chunks = n_my_tiles * NC;
 
     if (warp == 0) {
@@ -295,21 +309,21 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         // not all ask the same L2 lines for the same chunk at the same moment.
         if (lane == 0) {
             Ring<kW1Stages> r;
-            int cc = static_cast<int>(blockIdx.x) % NC;
+            int cc = cta % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
                 if (r.wrapped && !mbar_wait(&sm.w1_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM1 that read this slot is done
                 mbar_expect_tx(&sm.w1_full[r.slot], kTileBytes);
-                bulk_load(sm.w1[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes, kTileBytes, &sm.w1_full[r.slot]);
+                bulk_load(sm.w1[r.slot], p.packed + static_cast<size_t>(part * NC + cc) * kChunkBytes, kTileBytes, &sm.w1_full[r.slot]);
                 r.advance();
                 if (++cc == NC) cc = 0;
             }
         } else if (lane == 1) {
             Ring<kW2Stages> r;
-            int cc = static_cast<int>(blockIdx.x) % NC;
+            int cc = cta % NC;
             for (int g = 0; g < n_my_chunks; ++g) {
                 if (r.wrapped && !mbar_wait(&sm.w2_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM2 that read this slot is done
                 mbar_expect_tx(&sm.w2_full[r.slot], kTileBytes);
-                bulk_load(sm.w2[r.slot], p.packed + static_cast<size_t>(cc) * kChunkBytes + kTileBytes, kTileBytes, &sm.w2_full[r.slot]);
+                bulk_load(sm.w2[r.slot], p.packed + static_cast<size_t>(part * NC + cc) * kChunkBytes + kTileBytes, kTileBytes, &sm.w2_full[r.slot]);
                 r.advance();
                 if (++cc == NC) cc = 0;
             }
@@ -389,7 +403,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         // one copy per tree it touches.  Rows past the last token keep whatever the staging buffer held: a row of A
         // only feeds the same row of the output, which is not written.
         auto issue_tile_copy = [&](int it) {       // one lane
-            const int64_t tok0 = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(it) * gridDim.x) * kTok;
+            const int64_t tok0 = (static_cast<int64_t>(cta) + static_cast<int64_t>(it) * n_ctas) * kTok;
             int64_t remaining = p.n_tokens - tok0;
             if (remaining > kTok) remaining = kTok;
             mbar_expect_tx(&sm.stage_full, static_cast<uint32_t>(remaining) * (kCh * 4u));
@@ -453,13 +467,54 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.d2_empty[b]);
-            const int64_t q = (static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(t) * gridDim.x) * kTok + row;
+            const int64_t tile = static_cast<int64_t>(cta) + static_cast<int64_t>(t) * n_ctas;
+            const int64_t q = tile * kTok + row;
+            float4 val[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                val[j] = make_float4(0.5f * __uint_as_float(out[4 * j]), 0.5f * __uint_as_float(out[4 * j + 1]),
+                                     0.5f * __uint_as_float(out[4 * j + 2]), 0.5f * __uint_as_float(out[4 * j + 3]));
+            if (S > 1) {
+                // This CTA holds the sum over its share of the hidden dimension only.  Every part stores its tile; the
+                // part that draws the last ticket adds them up in part order (the host gives such a CTA one tile).
+                float4* mine = reinterpret_cast<float4*>(p.partials + ((tile * S + part) * kTok + row) * kCh + sub * 16u);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) __stcg(mine + j, val[j]);
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.part_done);
+                if (ew == 0) {
+                    const bool all_in = __all_sync(0xffffffffu, mbar_wait(&sm.part_done, 0u, abort_flag) ? 1 : 0) != 0;
+                    if (lane == 0) {
+                        int last = 0;
+                        if (all_in) {
+                            const unsigned int ticket = atomicAdd(&p.tickets[tile], 1u);
+                            last = ticket == static_cast<unsigned int>(S) - 1u;
+                            if (last) p.tickets[tile] = 0u;            // every part has arrived: ready for the next launch
+                        }
+                        sm.is_last_part = last;
+                        __threadfence();
+                        mbar_arrive(&sm.part_verdict);
+                    }
+                }
+                if (!__all_sync(0xffffffffu, mbar_wait(&sm.part_verdict, 0u, abort_flag) ? 1 : 0)) return false;
+                if (!*reinterpret_cast<volatile int*>(&sm.is_last_part)) return true;
+                __threadfence();
+#pragma unroll
+                for (int j = 0; j < 4; ++j) val[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int o = 0; o < S; ++o) {
+                    const float4* theirs = reinterpret_cast<const float4*>(p.partials + ((tile * S + o) * kTok + row) * kCh + sub * 16u);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 x = __ldcg(theirs + j);
+                        val[j].x += x.x; val[j].y += x.y; val[j].z += x.z; val[j].w += x.w;
+                    }
+                }
+            }
             if (q < p.n_tokens) {
                 float4* dst = reinterpret_cast<float4*>(p.v_out + q * kCh + sub * 16u);
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    dst[j] = make_float4(0.5f * __uint_as_float(out[4 * j]), 0.5f * __uint_as_float(out[4 * j + 1]),
-                                         0.5f * __uint_as_float(out[4 * j + 2]), 0.5f * __uint_as_float(out[4 * j + 3]));
+                for (int j = 0; j < 4; ++j) dst[j] = val[j];
             }
             return true;
         };
@@ -563,7 +618,8 @@ cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, 
 }
 
 cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
-                       const void* packed, int hidden, float* v_out, int32_t* status, cudaStream_t s) {
+                       const void* packed, int hidden, float* v_out, float* split_partials, unsigned int* split_tickets,
+                       int32_t* status, cudaStream_t s) {
     static bool configured[64] = {false};
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -588,7 +644,19 @@ cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_of
     if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     a.n_tiles = static_cast<int32_t>(tiles);
     a.status = status;
-    const int grid = a.n_tiles < sms ? a.n_tiles : sms;
+    // A frontier of fewer tiles than SMs is cut along the hidden dimension too, as far as the SMs (and the scratch) go.
+    a.split = 1;
+    a.partials = split_partials;
+    a.tickets = split_tickets;
+    if (split_partials && split_tickets) {
+        const int room = sms < kMlpSplitMaxCtas ? sms : kMlpSplitMaxCtas;
+        for (int cand = 8; cand > 1; cand >>= 1)
+            if (a.n_chunks % cand == 0 && static_cast<int64_t>(a.n_tiles) * cand <= room) {
+                a.split = cand;
+                break;
+            }
+    }
+    const int grid = a.split > 1 ? a.n_tiles * a.split : (a.n_tiles < sms ? a.n_tiles : sms);
     return launch_overlapped(mlp_velocity_kernel, grid, kMlpThreads, sizeof(MlpSmem) + 1024, s, a);
 }
 
