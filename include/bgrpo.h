@@ -162,7 +162,9 @@ bgrpo_status bgrpo_tree_logprob(bgrpo_tree* tree, int32_t step, const float* v_d
  * multiple of 128.  bgrpo_velocity_mlp_pack reorders the weights once into the tiled shared-memory image the kernel
  * streams (packed_dev: device, bgrpo_velocity_mlp_packed_bytes(hidden) bytes, 1024-byte aligned).
  * W1_bf16_dev: device [64][hidden] bf16 bits; W2_bf16_dev: device [hidden][64] bf16 bits.
- * v_out_dev: device [n_trees][W_i][D] float32. */
+ * v_out_dev: device [n_trees][W_i][D] float32.  Frontiers of fewer 128-token tiles than SMs are cut along the hidden
+ * dimension as well; the partial sums of that split live in the tree's scratch (the workspace query accounts for them)
+ * and are added in a fixed order, so repeated calls give identical bits. */
 size_t       bgrpo_velocity_mlp_packed_bytes(int32_t hidden);
 bgrpo_status bgrpo_velocity_mlp_pack(const uint16_t* W1_bf16_dev, const uint16_t* W2_bf16_dev, int32_t hidden,
                                      void* packed_dev, void* stream);
