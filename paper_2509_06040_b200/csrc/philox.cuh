@@ -68,13 +68,14 @@ __device__ __forceinline__ float fast_cos(float x) {
 //    and the sign change is absorbed into r.
 __device__ __forceinline__ float2 box_muller(uint32_t wa, uint32_t wb) {
     const float ua = uniform_open(wa);
-    const float ub = uniform_open(wb);
     const float w = 1.0f - ua;
     const float series = fmaf(w, w, w + w);
     const float viaLog = -1.3862944f * fast_log2(ua);          // -2 ln 2 * log2(u)
     const float r2 = (w < 0.001953125f) ? series : viaLog;
     const float nr = -fast_sqrt(r2);
-    const float th = fmaf(ub, 6.2831855f, -3.1415927f);       // 2 pi u_b - pi
+    // 2 pi u_b - pi with u_b = m - (1 - 2^-24), m in [1, 2) the float built from the word's top 23 bits: the constant
+    // term takes the subtraction in (its float32 rounding moves the angle by < 5e-7, i.e. xi by < 3e-6)
+    const float th = fmaf(__uint_as_float((wb >> 9) | 0x3f800000u), 6.2831855f, -9.4247776f);
     return make_float2(nr * fast_cos(th), nr * fast_sin(th));
 }
 

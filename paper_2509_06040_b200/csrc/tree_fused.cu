@@ -52,15 +52,16 @@ __device__ __forceinline__ void emit_child(const FusedLaunch& p, const Ctx& cx, 
             }
             c[k] = fma4(g, xi, m[k]);
             __stcs(row + cx.e[k], c[k]);
-            const float dx = c[k].x - m[k].x, dy = c[k].y - m[k].y, dz = c[k].z - m[k].z, dw = c[k].w - m[k].w;
-            acc = fmaf(dx, dx, acc);
-            acc = fmaf(dy, dy, acc);
-            acc = fmaf(dz, dz, acc);
-            acc = fmaf(dw, dw, acc);
+            // z' - mean is g xi up to the rounding of z': sum xi^2, times g^2 once per warp
+            acc = fmaf(xi.x, xi.x, acc);
+            acc = fmaf(xi.y, xi.y, acc);
+            acc = fmaf(xi.z, xi.z, acc);
+            acc = fmaf(xi.w, xi.w, acc);
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+    acc *= g * g;
     const int64_t r = cx.tree_row0 + child_local;
     if (cx.lane == 0) p.partialsf[r * p.per_row + cx.chunk * (kFusedThreads / 32) + cx.warp] = acc;
     if (cx.writes_table) {

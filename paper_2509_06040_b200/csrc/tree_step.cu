@@ -200,11 +200,20 @@ __device__ __forceinline__ void compute_tile(const StepLaunch& p, const float4 (
                 } else {
                     c = __ldcs(zc + static_cast<size_t>(b) * D4 + e);
                 }
-                const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
-                acc[b] = fmaf(dx, dx, acc[b]);
-                acc[b] = fmaf(dy, dy, acc[b]);
-                acc[b] = fmaf(dz, dz, acc[b]);
-                acc[b] = fmaf(dw, dw, acc[b]);
+                if (WRITE) {
+                    // z' - mean is g xi up to the rounding of z' (relative 6e-8 of |z'|, far below the 1e-5 the log-prob
+                    // is good to): sum xi^2 here, times g^2 once per warp below
+                    acc[b] = fmaf(xi[b].x, xi[b].x, acc[b]);
+                    acc[b] = fmaf(xi[b].y, xi[b].y, acc[b]);
+                    acc[b] = fmaf(xi[b].z, xi[b].z, acc[b]);
+                    acc[b] = fmaf(xi[b].w, xi[b].w, acc[b]);
+                } else {
+                    const float dx = c.x - m.x, dy = c.y - m.y, dz = c.z - m.z, dw = c.w - m.w;
+                    acc[b] = fmaf(dx, dx, acc[b]);
+                    acc[b] = fmaf(dy, dy, acc[b]);
+                    acc[b] = fmaf(dz, dz, acc[b]);
+                    acc[b] = fmaf(dw, dw, acc[b]);
+                }
             }
         }
     }
@@ -255,6 +264,7 @@ step_kernel(const __grid_constant__ StepLaunch p) {
         float f = acc[b];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) f += __shfl_down_sync(0xffffffffu, f, o);
+        if (WRITE) f *= p.g * p.g;
         if (lane == 0)
             p.partialsf[((tree_row0 + child0 + b) * p.nchunks + chunk) * kStepWarps + warp] = f;
     }
