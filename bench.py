@@ -42,12 +42,12 @@ NOMINAL_HBM_GBS = 8000.0
 # reported per launch is bytes-per-unit times the units of an average launch of the timed workload (traffic grows in
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
-    "step_kernel": {"workload": "video", "bytes": 75.601408e6 + 12.221184e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "2126f58c27b4"},
-    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.264832e6 + 214.634752e6, "units": 1036800,
-                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "f8c2d9ea6390"},
-    "rollout_fused_kernel": {"workload": "video", "bytes": 16.817664e6 + 865.891584e6, "units": 110 * 2096640,
-                             "sources": ("tree_fused.cu", "philox.cuh", "internal.h"), "source_hash": "bd5d30f37ce1"},
+    "step_kernel": {"workload": "video", "bytes": 75.591424e6 + 12.780800e6, "units": 8 * 2096640,
+                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "b9f579f780b1"},
+    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.370048e6 + 214.886912e6, "units": 1036800,
+                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "d870f89963fb"},
+    "rollout_fused_kernel": {"workload": "video", "bytes": 16.817152e6 + 866.309120e6, "units": 110 * 2096640,
+                             "sources": ("tree_fused.cu", "philox.cuh", "internal.h"), "source_hash": "5b1c4fdbdc7b"},
 }
 
 
