@@ -18,6 +18,7 @@ import argparse
 import hashlib
 import json
 import os
+import re
 import subprocess
 import sys
 import tempfile
@@ -43,11 +44,11 @@ NOMINAL_HBM_GBS = 8000.0
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
     "step_kernel": {"workload": "video", "bytes": 75.591424e6 + 12.780800e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh", "internal.h"), "source_hash": "b9f579f780b1"},
+                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d8106b7ec642"},
     "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.370048e6 + 214.886912e6, "units": 1036800,
-                            "sources": ("mlp_velocity.cu", "internal.h"), "source_hash": "d870f89963fb"},
+                            "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "1b67c54d890b"},
     "rollout_fused_kernel": {"workload": "video", "bytes": 16.817152e6 + 866.309120e6, "units": 110 * 2096640,
-                             "sources": ("tree_fused.cu", "philox.cuh", "internal.h"), "source_hash": "5b1c4fdbdc7b"},
+                             "sources": ("tree_fused.cu", "philox.cuh"), "shape": "kFused", "source_hash": "d109bb08cf93"},
 }
 
 
@@ -62,10 +63,17 @@ def load_peaks():
     return d
 
 
-def kernel_source_hash(names=("tree_step.cu", "philox.cuh", "internal.h")):
+def kernel_source_hash(names, shape=None):
+    """Hash of a kernel's own sources and of the lines of internal.h that define its launch shape (constants whose
+    name matches `shape`), so that an edit elsewhere in the shared header does not disown a still-valid capture."""
     h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2509_06040_b200", "csrc")
     for n in names:
-        h.update(open(os.path.join(ROOT, "paper_2509_06040_b200", "csrc", n), "rb").read())
+        h.update(open(os.path.join(csrc, n), "rb").read())
+    if shape:
+        for line in open(os.path.join(csrc, "internal.h")):
+            if line.startswith("constexpr") and re.search(shape, line):
+                h.update(line.encode())
     return h.hexdigest()[:12]
 
 
@@ -97,7 +105,7 @@ def step_children(w):
 def ncu_traffic(kernel, units_per_launch):
     """DRAM bytes of an average launch, scaled from the committed ncu capture; None once the kernel has changed."""
     tr = NCU_TRAFFIC[kernel]
-    if tr["source_hash"] != kernel_source_hash(tr["sources"]):
+    if tr["source_hash"] != kernel_source_hash(tr["sources"], tr.get("shape")):
         return None
     return tr["bytes"] / tr["units"] * units_per_launch
 

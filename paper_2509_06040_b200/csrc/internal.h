@@ -209,7 +209,7 @@ cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s);
 
 struct PruneLaunch {
     const float* rbar; const int32_t* table; uint8_t* mask;
-    LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes, mode, k, last_split, ignore_last; uint64_t pruned_bits;
+    LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes, mode, k, last_split, ignore_last, values_in_smem; uint64_t pruned_bits;
 };
 cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s);
 

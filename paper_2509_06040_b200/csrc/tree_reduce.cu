@@ -1,7 +1,7 @@
 // Tree reductions: reward fusion (Eq. 3) + depth-wise normalisation (Eq. 4) in one kernel, and the width / depth
 // pruning masks ("Pruning Strategies") in another.  A tree has at most a few thousand nodes, so one CTA owns one
 // tree, keeps the per-node state in shared memory as doubles and walks the levels; the kernels are latency-bound.
-// A tree whose per-node state does not fit in shared memory (more than 12 800 nodes: K = 4 with seven splits, say)
+// A tree whose per-node state does not fit in shared memory (more than about 8 500 nodes: K = 4 with seven splits, say)
 // keeps it in the caller's scratch instead; the code is the same, only the pointer differs.
 //
 // Fusion uses the bottom-up form of Eq. 3.  With a_c = beta*logp(c) the softmax weight of leaf l under node n
@@ -25,9 +25,10 @@ __global__ void __launch_bounds__(kTreeThreads)
 fuse_advantage_kernel(const FuseLaunch p) {
     extern __shared__ double sm[];
     const int tree = blockIdx.x;
-    const bool in_smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double) <= kTreeSmemLimit;
+    const bool in_smem = static_cast<size_t>(p.nodes) * 3 * sizeof(double) <= kTreeSmemLimit;
     double* rb = in_smem ? sm : p.node_scratch + static_cast<int64_t>(tree) * 2 * p.nodes_cap;   // rbar per node
     double* ls = rb + (in_smem ? p.nodes : p.nodes_cap);                                          // log S per node
+    double* la = in_smem ? ls + p.nodes : nullptr;     // beta * logp per node, fetched once (a level then waits for no global load)
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     const int T = p.T;
     const int leaves = p.lv.width[T];
@@ -35,6 +36,9 @@ fuse_advantage_kernel(const FuseLaunch p) {
     __shared__ int bad;
     if (threadIdx.x == 0) bad = 0;
     __syncthreads();
+    const double beta = p.beta_scaled;
+    if (la)
+        for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) la[n] = beta * static_cast<double>(p.logp[row0 + n]);
     for (int l = threadIdx.x; l < leaves; l += kTreeThreads) {
         const float r = p.leaf_r[static_cast<int64_t>(tree) * leaves + l];
         if (!isfinite(r)) bad = 1;
@@ -43,7 +47,6 @@ fuse_advantage_kernel(const FuseLaunch p) {
     }
     __syncthreads();
     if (bad && threadIdx.x == 0) atomicOr(p.status, 1);
-    const double beta = p.beta_scaled;
     for (int d = T - 1; d >= 0; --d) {
         const int fan = p.lv.fanout[d];
         const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
@@ -54,7 +57,7 @@ fuse_advantage_kernel(const FuseLaunch p) {
 #pragma unroll
             for (int b = 0; b < BGRPO_MAX_K; ++b) {
                 if (b < fan) {
-                    a[b] = beta * static_cast<double>(p.logp[row0 + c0 + b]) + ls[c0 + b];
+                    a[b] = (la ? la[c0 + b] : beta * static_cast<double>(p.logp[row0 + c0 + b])) + ls[c0 + b];
                     m = fmax(m, a[b]);
                 }
             }
@@ -151,11 +154,17 @@ __device__ __forceinline__ bool beats(float v_other, int i_other, float v_me, in
 
 __global__ void __launch_bounds__(kTreeThreads)
 prune_kernel(const PruneLaunch p) {
-    extern __shared__ unsigned char keep[];            // per node
+    extern __shared__ unsigned char keep[];            // per node, then (small trees) the node values as floats
     const int tree = blockIdx.x;
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     const int T = p.T;
     const float* rbar = p.rbar + row0;
+    if (p.values_in_smem) {        // fetched once: a level then waits for no global load
+        float* vals = reinterpret_cast<float*>(keep + ((static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15)));
+        for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) vals[n] = rbar[n];
+        rbar = vals;
+        __syncthreads();
+    }
     if (p.mode == BGRPO_WIDTH_EXTREME_B) {
         for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) keep[n] = 0;
         __syncthreads();
@@ -263,7 +272,7 @@ cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s) {
 }
 
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
-    size_t smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double);
+    size_t smem = static_cast<size_t>(p.nodes) * 3 * sizeof(double);
     if (smem > kTreeSmemLimit) smem = 0;          // per-node state in the caller's scratch
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(fuse_advantage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
@@ -273,8 +282,11 @@ cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s) {
-    const size_t smem = (static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15);
+cudaError_t launch_prune(const PruneLaunch& p0, cudaStream_t s) {
+    PruneLaunch p = p0;
+    size_t smem = (static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15);
+    p.values_in_smem = smem + static_cast<size_t>(p.nodes) * sizeof(float) <= kTreeSmemLimit ? 1 : 0;
+    if (p.values_in_smem) smem += static_cast<size_t>(p.nodes) * sizeof(float);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
