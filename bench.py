@@ -248,6 +248,7 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
     t_step = np.zeros(w.T)
     t_mlp = np.zeros(w.T)
     t_other = 0.0
+    t_tail = np.zeros(3)          # leaf rewards, fusion + advantages, pruning masks
 
     def evs(n):
         return [torch.cuda.Event(enable_timing=True) for _ in range(n)]
@@ -269,19 +270,24 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
             e_lvl[i][1].record()
             B.tree_step(s.tree, 1 if i in w.splits else 0, s.v if w.velocity == "mlp" else None)
             e_lvl[i][2].record()
+        e_red = evs(2)
         e_tail[0].record()
         s.rewards()
+        e_red[0].record()
         s.fuse_advantage()
+        e_red[1].record()
         s.prune()
         e_tail[1].record()
         torch.cuda.synchronize()
         t_other += e_init[0].elapsed_time(e_init[1]) + e_tail[0].elapsed_time(e_tail[1])
+        t_tail += np.array([e_tail[0].elapsed_time(e_red[0]), e_red[0].elapsed_time(e_red[1]), e_red[1].elapsed_time(e_tail[1])])
         for i in range(w.T):
             t_mlp[i] += e_lvl[i][0].elapsed_time(e_lvl[i][1]) if w.velocity == "mlp" else 0.0
             t_step[i] += e_lvl[i][1].elapsed_time(e_lvl[i][2])
     t_step /= reps
     t_mlp /= reps
     t_other /= reps
+    t_tail /= reps
     sb = np.array(step_bytes_per_launch(w, w.n_trees), dtype=np.float64)
     step_gbs = sb.sum() / (t_step.sum() * 1e-3) / 1e9
     widest = int(np.argmax(sb))
@@ -293,7 +299,12 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
                  "widest_launch": {"step": widest, "bytes": float(sb[widest]), "ms": float(t_step[widest]),
                                    "gbs": float(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
                  "traffic": ncu_traffic("step_kernel", float(sum(c * w.D for c in step_children(w))) / w.T)}
-    breakdown = {"step_ms": float(t_step.sum()), "mlp_ms": float(t_mlp.sum()), "other_ms": float(t_other)}
+    reward_bytes = 0.0 if w.reward == "mixture" else float(w.n_trees * (w.leaves + 1) * 4 * w.D)   # leaf rows once, target once per tree
+    breakdown = {"step_ms": float(t_step.sum()), "mlp_ms": float(t_mlp.sum()), "other_ms": float(t_other),
+                 "leaf_reward_ms": float(t_tail[0]), "fuse_advantage_ms": float(t_tail[1]), "prune_ms": float(t_tail[2]),
+                 "leaf_reward_gbs": (reward_bytes / (t_tail[0] * 1e-3) / 1e9) if reward_bytes and t_tail[0] > 0 else None,
+                 "note": "intervals between in-stream events: each holds one launch and its launch gap; the reduction "
+                         "kernels handle a few hundred scalars per tree and are latency-bound"}
     roof = roof_step
     if w.velocity == "mlp" and t_mlp.sum() > t_step.sum():
         fl = np.array(mlp_flops_per_launch(w, w.n_trees), dtype=np.float64)
