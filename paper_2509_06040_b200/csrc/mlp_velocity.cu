@@ -63,7 +63,7 @@ struct MlpSmem {
     alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
     alignas(1024) float stage[kTok * kCh];                   // float32 latents of the next tile, as they are in global memory
     unsigned long long w1_full[kW1Stages], w1_free[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
-    unsigned long long stage_full, a_full[2], a_empty[2], d1_full[2], d1_empty[2], h_full[2], h_free[2], d2_full[2], d2_empty[2];
+    unsigned long long stage_full, first_a, a_full[2], a_empty[2], d1_full[2], d1_empty[2], h_full[2], h_free[2], d2_full[2], d2_empty[2];
     unsigned long long part_done, part_verdict;   // split mode: all epilogue warps have stored their partials / the ticket is drawn
     int is_last_part;
     uint32_t tmem_base;
@@ -235,6 +235,21 @@ __device__ __forceinline__ float gelu_x2(float x) {
 // byte offset of the 16-byte piece `c16` of row r inside a 128-byte-swizzled tile of 128-byte rows
 __device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c16) { return r * 128u + ((c16 ^ (r & 7u)) << 4); }
 
+// Converts rows [r_begin, r_end) of the float32 staging tile to the bf16 K-major swizzled A tile; one warp, two rows per
+// step (16 lanes x 16 bytes cover a row).
+__device__ __forceinline__ void convert_rows(const float* stage, unsigned char* atile, int r_begin, int r_end, int lane) {
+    const uint32_t c4 = static_cast<uint32_t>(lane & 15);
+#pragma unroll 8
+    for (int r0 = r_begin; r0 < r_end; r0 += 2) {
+        const uint32_t r = static_cast<uint32_t>(r0 + (lane >> 4));
+        const float4 zv = *reinterpret_cast<const float4*>(stage + r * kCh + c4 * 4u);
+        uint2 packed2;
+        packed2.x = pack_bf16(zv.x, zv.y);
+        packed2.y = pack_bf16(zv.z, zv.w);
+        *reinterpret_cast<uint2*>(atile + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
+    }
+}
+
 struct MlpArgs {
     const float* latents;     // pool base
     int64_t tree_stride;      // elements between trees in the pool
@@ -269,6 +284,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             mbar_init(&sm.w2_free[q], 1);
         }
         mbar_init(&sm.stage_full, 1);
+        mbar_init(&sm.first_a, kEpiWarps);
         mbar_init(&sm.part_done, kEpiWarps);
         mbar_init(&sm.part_verdict, 1);
         for (int q = 0; q < 2; ++q) {
@@ -423,22 +439,19 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         if (n_my_tiles > 0 && lane == 0) issue_tile_copy(0);
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int ab = it & 1;
-            ok = mbar_wait(&sm.stage_full, static_cast<uint32_t>(it) & 1u, abort_flag);
-            if (ok && it >= 2) ok = mbar_wait(&sm.a_empty[ab], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
-            if (!ok) break;
-            const uint32_t c4 = static_cast<uint32_t>(lane & 15);            // float4 index within the row; the warp covers 2 rows per step
-            unsigned char* atile = sm.a[ab];
-#pragma unroll 8
-            for (int r0 = 0; r0 < kTok; r0 += 2) {
-                const uint32_t r = static_cast<uint32_t>(r0 + (lane >> 4));
-                const float4 zv = *reinterpret_cast<const float4*>(sm.stage + r * kCh + c4 * 4u);
-                uint2 packed2;
-                packed2.x = pack_bf16(zv.x, zv.y);
-                packed2.y = pack_bf16(zv.z, zv.w);
-                *reinterpret_cast<uint2*>(atile + sw128(r, c4 >> 1) + (c4 & 1u) * 8u) = packed2;
+            if (it == 0) {
+                // The first tile is on the critical path of the launch and the sixteen epilogue warps have nothing to do
+                // yet: they convert it, eight rows each (one warp needs about 2 us for a tile), and report here.
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.first_a, 0u, abort_flag) ? 1 : 0) != 0;
+                if (!ok) break;
+            } else {
+                ok = mbar_wait(&sm.stage_full, static_cast<uint32_t>(it) & 1u, abort_flag);
+                if (ok && it >= 2) ok = mbar_wait(&sm.a_empty[ab], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+                if (!ok) break;
+                convert_rows(sm.stage, sm.a[ab], 0, kTok, lane);
+                proxy_fence();
             }
-            proxy_fence();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(&sm.a_full[ab]);
@@ -455,6 +468,15 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         const uint32_t lane_addr = (quarter * 32u) << 16;
         bool ok = true;
         int next_out = 0;             // first tile this warp has not written out yet
+        if (n_my_tiles > 0) {         // this warp's eight rows of the first A tile (see the loader warp)
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.stage_full, 0u, abort_flag) ? 1 : 0) != 0;
+            if (ok) {
+                convert_rows(sm.stage, sm.a[0], ew * (kTok / kEpiWarps), (ew + 1) * (kTok / kEpiWarps), lane);
+                proxy_fence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.first_a);
+            }
+        }
 
         // v = 0.5 D2 of tile t (this warp's 32 rows x 16 channels)
         auto output_tile = [&](int t) -> bool {
