@@ -526,16 +526,29 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
                 const float4* parts = reinterpret_cast<const float4*>(p.partials) + tile * S * (kTok * kCh / 4);
                 float4* vt = reinterpret_cast<float4*>(p.v_out) + tile * (kTok * kCh / 4);
                 const int64_t rows_left = p.n_tokens - tile * kTok;
-                for (int i = 0; i < (kTok * kCh / 4) / (kEpiWarps * 32); ++i) {
-                    const int idx = i * (kEpiWarps * 32) + ew * 32 + lane;
-                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int o = 0; o < S; o += 2) {       // S is even: added in part order, two loads in flight
-                        const float4 x0 = __ldcg(parts + static_cast<int64_t>(o) * (kTok * kCh / 4) + idx);
-                        const float4 x1 = __ldcg(parts + static_cast<int64_t>(o + 1) * (kTok * kCh / 4) + idx);
-                        sum.x += x0.x; sum.y += x0.y; sum.z += x0.z; sum.w += x0.w;
-                        sum.x += x1.x; sum.y += x1.y; sum.z += x1.z; sum.w += x1.w;
+                constexpr int kPer = (kTok * kCh / 4) / (kEpiWarps * 32);      // float4 per thread: 4
+                constexpr int64_t kTile4 = kTok * kCh / 4;
+                float4 sum[kPer];
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) sum[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int idx0 = ew * 32 + lane;
+                for (int o = 0; o < S; o += 2) {       // S is even: parts added in order, eight loads in flight
+                    float4 x[2][kPer];
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        x[0][i] = __ldcg(parts + static_cast<int64_t>(o) * kTile4 + idx0 + i * (kEpiWarps * 32));
+                        x[1][i] = __ldcg(parts + static_cast<int64_t>(o + 1) * kTile4 + idx0 + i * (kEpiWarps * 32));
                     }
-                    if (idx / (kCh / 4) < rows_left) vt[idx] = sum;
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        sum[i].x += x[0][i].x; sum[i].y += x[0][i].y; sum[i].z += x[0][i].z; sum[i].w += x[0][i].w;
+                        sum[i].x += x[1][i].x; sum[i].y += x[1][i].y; sum[i].z += x[1][i].z; sum[i].w += x[1][i].w;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    const int idx = idx0 + i * (kEpiWarps * 32);
+                    if (idx / (kCh / 4) < rows_left) vt[idx] = sum[i];
                 }
                 return true;
             }
