@@ -289,13 +289,38 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
     t_other /= reps
     t_tail /= reps
     sb = np.array(step_bytes_per_launch(w, w.n_trees), dtype=np.float64)
-    step_gbs = sb.sum() / (t_step.sum() * 1e-3) / 1e9
+    step_gbs_events = sb.sum() / (t_step.sum() * 1e-3) / 1e9
+    step_ms_group = None
+    if w.velocity == "linear":
+        # With the closed-form velocity the T step launches follow one another with nothing in between: one pair of events
+        # around the group gives their average duration without the gap that an event between two launches costs.
+        tot = 0.0
+        for rep in range(reps):
+            if flush_buf is not None:
+                flush_buf.fill_(1.0)
+            s.init(seed=w.seed + 4000 + rep)
+            g0, g1 = evs(2)
+            g0.record()
+            for i in range(w.T - 1):      # the last step also enqueues the log-prob flush kernel: timed per launch above
+                B.tree_step(s.tree, 1 if i in w.splits else 0, None)
+            g1.record()
+            B.tree_step(s.tree, 1 if (w.T - 1) in w.splits else 0, None)
+            torch.cuda.synchronize()
+            tot += g0.elapsed_time(g1)
+        step_ms_group = tot / reps
+    if step_ms_group is not None:
+        step_gbs = sb[:-1].sum() / (step_ms_group * 1e-3) / 1e9
+    else:
+        step_gbs = step_gbs_events
     widest = int(np.argmax(sb))
     hbm_peak = float(peaks["hbm_gbs"])
     roof_step = {"bound": "hbm", "kernel": "step_kernel", "achieved": step_gbs, "peak": hbm_peak, "unit": "GB/s",
                  "frac": step_gbs / hbm_peak, "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
                  "peak_source": peaks["_source"], "launches_per_pass": w.T,
                  "bytes_per_pass": float(sb.sum()), "ms_per_pass": float(t_step.sum()),
+                 "timing": ("steps 0..T-2 back to back between one pair of events (%.4f ms for %.0f bytes)" % (step_ms_group, sb[:-1].sum()))
+                           if step_ms_group is not None else "one pair of events per launch",
+                 "gbs_with_an_event_between_launches": step_gbs_events,
                  "widest_launch": {"step": widest, "bytes": float(sb[widest]), "ms": float(t_step[widest]),
                                    "gbs": float(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
                  "traffic": ncu_traffic("step_kernel", float(sum(c * w.D for c in step_children(w))) / w.T)}
