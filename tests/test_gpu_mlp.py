@@ -143,3 +143,29 @@ def test_small_frontier_split_is_reproducible_and_agrees_with_the_unsplit_kernel
     ref = b.v.view(-1)[:small.D]
     rms = ref.pow(2).mean().sqrt().item()
     assert (outs[0] - ref).abs().max().item() <= 1e-5 * rms + 1e-6 * ref.abs().max().item()
+
+
+def test_repeated_passes_are_bit_identical(B):
+    """The whole path twice with the same seed, and once more after a pass with another seed in between: every output
+    is identical bit for bit.  Sums are taken in fixed orders and kernels that overlap on the stream (programmatic
+    dependent launch, the split of small MLP frontiers) wait for what they depend on."""
+    from paper_2509_06040_b200.session import TreeSession
+    w = Workload(name="mlp_repeat", n_trees=2, tokens=333, channels=64, T=6, K=2, splits=(0, 2, 3), sigma=0.3,
+                 velocity="mlp", reward="normal_plus_cos", hidden=512, width_mode=1, width_k=1)
+    inp = make_inputs(w)
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+
+    def snapshot(seed):
+        s.run_all(seed=seed)
+        torch.cuda.synchronize()
+        B.tree_sync_status(s.tree)
+        return [t.clone() for t in (s.latents, s.logp, s.rbar, s.adv, s.mask, s.node_table, s.leaf_r)]
+
+    first = snapshot(11)
+    second = snapshot(11)
+    other = snapshot(12)
+    third = snapshot(11)
+    for a, b, c in zip(first, second, third):
+        assert torch.equal(a, b) and torch.equal(a, c)
+    assert not torch.equal(first[0], other[0])
