@@ -45,8 +45,8 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_TRAFFIC = {
     "step_kernel": {"workload": "video", "bytes": 75.591424e6 + 12.780800e6, "units": 8 * 2096640,
                     "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d8106b7ec642"},
-    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.370048e6 + 214.886912e6, "units": 1036800,
-                            "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "1b67c54d890b"},
+    "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.295808e6 + 214.387712e6, "units": 1036800,
+                            "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "2141aa3f7a6b"},
     "rollout_fused_kernel": {"workload": "video", "bytes": 16.817152e6 + 866.309120e6, "units": 110 * 2096640,
                              "sources": ("tree_fused.cu", "philox.cuh"), "shape": "kFused", "source_hash": "d109bb08cf93"},
 }

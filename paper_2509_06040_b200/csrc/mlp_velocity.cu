@@ -24,7 +24,8 @@
 //                  two chunks after its last GEMM2 was issued, when it has long completed);
 //     warp 18      brings the NEXT tile's latents in with bulk asynchronous copies (one per tree the tile touches) into
 //                  a float32 staging buffer and converts them to the bf16 A tile while the current tile computes.  (Plain
-//                  loads from one warp kept only 4 KiB in flight and took longer per tile than the arithmetic.)
+//                  loads from one warp kept only 4 KiB in flight and took longer per tile than the arithmetic.)  The
+//                  first tile of a launch is converted by the sixteen epilogue warps, idle until then.
 // Shared-memory operands are K-major tiles of 128-byte rows in the 128-byte-swizzle layout the MMA descriptors
 // address; the weights are reordered once into exactly that image (bgrpo_velocity_mlp_pack), so a chunk arrives with
 // one copy per matrix.  No cluster multicast is used anywhere.
@@ -45,7 +46,7 @@ constexpr int kCh = 64;                   // channels = K of GEMM1 = N of GEMM2
 constexpr int kHc = 128;                  // hidden chunk = N of GEMM1 = K of GEMM2
 constexpr int kW1Stages = 3;               // W1 slot q is free again when the GEMM1 that read it has completed
 constexpr int kW2Stages = 4;               // W2 slot q is free again when the GEMM2 that read it has completed
-constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 32 columns of a chunk each
+constexpr int kEpiWarps = 16;             // two groups of eight: two warps per TMEM lane quarter, 64 columns of a chunk each
 constexpr int kLoaderWarp = 2 + kEpiWarps;
 constexpr int kGemm2Warp = 3 + kEpiWarps;
 constexpr int kMlpThreads = (4 + kEpiWarps) * 32;
