@@ -56,3 +56,48 @@ def test_video_config_whole_workload(B):
     assert int(mask.sum()) == sum(1 for n in range(1, topo.nodes) if mask[n])
     # top-1 per split keeps exactly one leaf
     assert int(mask[list(topo.leaf_ids())].sum()) == 1
+
+
+@pytest.mark.parametrize("name,depth", [("image", 0), ("image", 10), ("image_batch", 10), ("group", 12)])
+def test_mlp_stage_full_size_sampled(B, name, depth):
+    """The MLP velocity stage at the benchmark's sizes and launch shapes: the root level of the single image tree (16
+    tiles, cut 8 ways along the hidden dimension), its widest level (254 tiles on 148 SMs), the widest level of the
+    32-tree batch (8100 tiles) and of the 8-tree group workload.  The frontier is filled with seeded normal latents; a
+    sample of tokens (tile heads and tails, tree and node boundaries, the ragged last tile, random ones) is compared with
+    the oracle's bf16-emulating MLP, token by token."""
+    from oracle import mlp
+    from paper_2509_06040_b200.session import TreeSession
+    w = CONFIGS[name]
+    inp = make_inputs(w)
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+    s.init()
+    s.v.zero_()
+    for i in range(depth):                       # grow the tree to the depth under test; the latents are replaced below
+        B.tree_step(s.tree, 1 if i in w.splits else 0, s.v)
+    widths, offs = B.tree_levels(s.tree)
+    W, off = widths[depth], offs[depth]
+    rng = np.random.default_rng([7, depth, w.n_trees])
+    z = rng.standard_normal((w.n_trees, W, w.D), dtype=np.float32)
+    s.latents[:, off:off + W].copy_(torch.from_numpy(z))
+    s.v.fill_(float("nan"))
+    B.velocity_mlp(s.tree, s.packed, w.hidden, s.v)
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    n_tok = w.n_trees * W * w.tokens
+    got = s.v.view(-1)[:n_tok * 64].view(n_tok, 64)
+    zt = z.reshape(n_tok, 64)
+    per_tree = W * w.tokens
+    picks = set(range(0, 130)) | set(range(n_tok - 130, n_tok)) | {int(x) for x in rng.integers(0, n_tok, 400)}
+    for t in range(1, min(w.n_trees, 3)):        # around tree boundaries
+        picks |= set(range(t * per_tree - 3, t * per_tree + 3))
+    for j in range(1, min(W, 3)):                # around node boundaries
+        picks |= set(range(j * w.tokens - 3, j * w.tokens + 3))
+    for tile in (1, 2, (n_tok // 128) // 2):     # heads and tails of some tiles
+        picks |= set(range(tile * 128 - 2, tile * 128 + 2))
+    idx = np.array(sorted(p for p in picks if 0 <= p < n_tok))
+    ref = mlp.mlp_velocity(zt[idx], inp.W1, inp.W2)
+    out = got[torch.from_numpy(idx).cuda()].cpu().numpy()
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    assert np.all(np.abs(out - ref) <= 2e-2 * np.abs(ref) + 2e-2 * rms), float(np.abs(out - ref).max() / rms)
+    assert not torch.isnan(got).any()            # every token of the frontier was written
