@@ -101,3 +101,55 @@ def test_mlp_stage_full_size_sampled(B, name, depth):
     rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
     assert np.all(np.abs(out - ref) <= 2e-2 * np.abs(ref) + 2e-2 * rms), float(np.abs(out - ref).max() / rms)
     assert not torch.isnan(got).any()            # every token of the frontier was written
+
+
+@pytest.mark.parametrize("name,depth", [("image_batch", 9), ("image_batch", 10), ("group", 12)])
+def test_step_kernel_full_size_sampled_rows(B, name, depth):
+    """tree_step with a supplied velocity at the benchmark's widest launches (a split step and a non-split one of the
+    32-tree batch, the 64-wide level of the group workload): frontier latents and velocities are seeded normals, and for
+    a sample of (tree, parent) pairs - first, last, around the middle - every element of every child row and the
+    children's log-probs are compared with the oracle's Euler-Maruyama step (Eq. 2) on the same inputs."""
+    from oracle import philox, sde
+    from paper_2509_06040_b200.session import TreeSession
+    w = CONFIGS[name]
+    s = TreeSession(w)
+    s.upload_inputs(make_inputs(w))
+    s.init()
+    s.v.zero_()
+    for i in range(depth):
+        B.tree_step(s.tree, 1 if i in w.splits else 0, s.v)
+    widths, offs = B.tree_levels(s.tree)
+    W, off = widths[depth], offs[depth]
+    rng = np.random.default_rng([11, depth, w.n_trees])
+    z = rng.standard_normal((w.n_trees, W, w.D), dtype=np.float32)
+    v = rng.standard_normal((w.n_trees, W, w.D), dtype=np.float32)
+    s.latents[:, off:off + W].copy_(torch.from_numpy(z))
+    v_dev = s.v.view(-1)[:z.size].view(z.shape)
+    v_dev.copy_(torch.from_numpy(v))
+    split = depth in w.splits
+    B.tree_step(s.tree, 1 if split else 0, v_dev)
+    # the step's own log-prob sums are completed by the next call on the stream: here the recompute under the same
+    # velocity, which must give the same numbers (rho = 1)
+    again = torch.zeros_like(s.logp)
+    B.tree_logprob(s.tree, depth, v_dev, again)
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    widths, offs = B.tree_levels(s.tree)
+    off_c, fan = offs[depth + 1], (w.K if split else 1)
+    grid = w.t_grid().astype(np.float64)
+    t, h, sigma = float(grid[depth]), float(grid[depth] - grid[depth + 1]), f32(w.sigma)
+    g = sde.noise_scale(sigma, h)
+    logp = s.logp.cpu().numpy()
+    for tree, j in ((0, 0), (w.n_trees - 1, W - 1), (w.n_trees // 2, W // 2), (1, 1)):
+        mean = sde.em_mean(z[tree, j].astype(np.float64), v[tree, j].astype(np.float64), t, h, sigma)
+        for b in range(fan):
+            c = off_c + j * fan + b
+            eta = philox.node_noise(w.seed, tree * s.nodes_cap + c, depth, philox.TAG_INNOV, w.D)
+            child = (mean + g * eta).astype(np.float32)           # the workloads run with independent children (s = inf)
+            got = s.latents[tree, c].cpu().numpy()
+            assert np.abs(got - child).max() <= LATENT_TOL, (tree, j, b)
+            assert abs(logp[tree, c] - sde.transition_logp(child, mean, g)) <= LOGP_TOL
+            assert abs(float(again[tree, c]) - sde.transition_logp(child, mean, g)) <= LOGP_TOL
+    tab = s.node_table.cpu().numpy().reshape(4, w.n_trees, s.nodes_cap)
+    assert np.array_equal(tab[0, 0, off_c:off_c + W * fan], off + np.arange(W * fan) // fan)
+    assert np.all(tab[1, :, off_c:off_c + W * fan] == depth + 1)
