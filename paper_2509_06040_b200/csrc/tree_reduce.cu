@@ -52,6 +52,11 @@ fuse_advantage_kernel(const FuseLaunch p) {
         const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
         for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads) {
             const int c0 = offc + j * fan;
+            if (fan == 1) {      // an only child: its value is the parent's, and log S just picks up the edge
+                rb[off + j] = rb[c0];
+                ls[off + j] = (la ? la[c0] : beta * static_cast<double>(p.logp[row0 + c0])) + ls[c0];
+                continue;
+            }
             double a[BGRPO_MAX_K];
             double m = -INFINITY;
 #pragma unroll
@@ -189,26 +194,36 @@ prune_kernel(const PruneLaunch p) {
         (void)rows;
         __syncthreads();
     } else {
-        if (threadIdx.x == 0) keep[0] = 1;
+        // Top-k modes: a node is kept iff, at every ranked split on its root path, the ancestor (or the node itself)
+        // ranks among the k best of its siblings.  Every node walks its own path (children of the j-th node of depth d
+        // are j*F + b of depth d+1, so the parent of j is j / F): no level-by-level pass, no barrier.
+        __shared__ int s_off[BGRPO_MAX_T + 2], s_fan[BGRPO_MAX_T];
+        for (int i = threadIdx.x; i <= T + 1; i += kTreeThreads) s_off[i] = p.lv.offset[i];
+        for (int i = threadIdx.x; i < T; i += kTreeThreads) s_fan[i] = p.lv.fanout[i];
         __syncthreads();
-        for (int d = 0; d < T; ++d) {
-            const int fan = p.lv.fanout[d];
-            const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
-            const bool ranked = fan > 1 && (p.mode == BGRPO_WIDTH_PER_SPLIT_TOPK ||
-                                            (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && d == p.last_split));
-            for (int c = threadIdx.x; c < p.lv.width[d + 1]; c += kTreeThreads) {
-                const int j = c / fan, b = c - j * fan;
-                unsigned char k = keep[off + j];
+        for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) {       // one node per thread, all depths at once
+            int d = 0;
+            while (d < T && n >= s_off[d + 1]) ++d;
+            const bool depth_ok = d > 0 && !((p.pruned_bits >> (d - 1)) & 1ull) && !(p.ignore_last && d == T);
+            bool kept = true;
+            int j = n - s_off[d];
+            for (int e = d; e > 0 && kept; --e) {                // e: depth of the node j on the path
+                const int fan = s_fan[e - 1];
+                const int pj = j / fan, b = j - pj * fan;
+                const bool ranked = fan > 1 && (p.mode == BGRPO_WIDTH_PER_SPLIT_TOPK ||
+                                                (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && e - 1 == p.last_split));
                 if (ranked) {
-                    const float v = rbar[offc + c];
+                    const int sib0 = s_off[e] + pj * fan;
+                    const float v = rbar[sib0 + b];
                     int rank = 0;
-                    for (int q = 0; q < fan; ++q) rank += beats(rbar[offc + j * fan + q], q, v, b) ? 1 : 0;
-                    k = (k && rank < p.k) ? 1 : 0;
+                    for (int q = 0; q < fan; ++q) rank += beats(rbar[sib0 + q], q, v, b) ? 1 : 0;
+                    kept = rank < p.k;
                 }
-                keep[offc + c] = k;
+                j = pj;
             }
-            __syncthreads();
+            p.mask[row0 + n] = (depth_ok && kept) ? 1 : 0;
         }
+        return;
     }
     for (int d = 0; d <= T; ++d) {
         const bool depth_ok = d > 0 && !((p.pruned_bits >> (d - 1)) & 1ull) && !(p.ignore_last && d == T);
