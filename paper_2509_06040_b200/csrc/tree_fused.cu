@@ -117,6 +117,8 @@ __device__ __forceinline__ void walk(const FusedLaunch& p, const Ctx& cx, int i,
 template <int MAXS, bool SHARED>
 __global__ void __launch_bounds__(kFusedThreads)
 rollout_fused_kernel(const __grid_constant__ FusedLaunch p) {
+    pdl_release();
+    pdl_wait();
     Ctx cx;
     cx.chunk = blockIdx.x % p.nchunks;
     const int tree = blockIdx.x / p.nchunks;
@@ -148,6 +150,8 @@ rollout_fused_kernel(const __grid_constant__ FusedLaunch p) {
 // throughout.
 __global__ void __launch_bounds__(256)
 finalize_tree_kernel(const __grid_constant__ FusedLaunch p, int32_t nodes) {
+    pdl_release();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int64_t w = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t total = static_cast<int64_t>(p.n_trees) * (nodes - 1);
@@ -179,18 +183,17 @@ cudaError_t launch_rollout_fused(const FusedLaunch& p, int32_t nodes, cudaStream
     const unsigned int grid = static_cast<unsigned int>(items);
     const int n_splits = __builtin_popcountll(p.split_bits);
     if (n_splits > kFusedMaxSplits) return cudaErrorInvalidValue;
+    cudaError_t e;
     if (p.shared_noise) {
-        if (n_splits <= 3) rollout_fused_kernel<3, true><<<grid, kFusedThreads, 0, s>>>(p);
-        else rollout_fused_kernel<kFusedMaxSplits, true><<<grid, kFusedThreads, 0, s>>>(p);
+        if (n_splits <= 3) e = launch_overlapped(rollout_fused_kernel<3, true>, grid, kFusedThreads, 0, s, p);
+        else e = launch_overlapped(rollout_fused_kernel<kFusedMaxSplits, true>, grid, kFusedThreads, 0, s, p);
     } else {
-        if (n_splits <= 3) rollout_fused_kernel<3, false><<<grid, kFusedThreads, 0, s>>>(p);
-        else rollout_fused_kernel<kFusedMaxSplits, false><<<grid, kFusedThreads, 0, s>>>(p);
+        if (n_splits <= 3) e = launch_overlapped(rollout_fused_kernel<3, false>, grid, kFusedThreads, 0, s, p);
+        else e = launch_overlapped(rollout_fused_kernel<kFusedMaxSplits, false>, grid, kFusedThreads, 0, s, p);
     }
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || nodes < 2) return e;
     const int64_t warps = static_cast<int64_t>(p.n_trees) * (nodes - 1);
-    finalize_tree_kernel<<<static_cast<unsigned int>((warps + 7) / 8), 256, 0, s>>>(p, nodes);
-    return cudaGetLastError();
+    return launch_overlapped(finalize_tree_kernel, static_cast<unsigned int>((warps + 7) / 8), 256, 0, s, p, nodes);
 }
 
 }  // namespace bgrpo

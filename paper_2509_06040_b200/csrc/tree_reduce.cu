@@ -23,6 +23,8 @@ __device__ __forceinline__ double warp_sum_d(double x) {
 
 __global__ void __launch_bounds__(kTreeThreads)
 fuse_advantage_kernel(const FuseLaunch p) {
+    pdl_release();
+    pdl_wait();
     extern __shared__ double sm[];
     const int tree = blockIdx.x;
     const bool in_smem = static_cast<size_t>(p.nodes) * 3 * sizeof(double) <= kTreeSmemLimit;
@@ -105,6 +107,8 @@ fuse_advantage_kernel(const FuseLaunch p) {
 //   log S_n = logsumexp_c(a_c + log S_c),   log Q_n = logsumexp_c(2 a_c + log Q_c),   ESS = exp(2 log S - log Q).
 __global__ void __launch_bounds__(kTreeThreads)
 fusion_ess_kernel(const EssLaunch p) {
+    pdl_release();
+    pdl_wait();
     extern __shared__ double sm[];
     const int tree = blockIdx.x;
     const bool in_smem = static_cast<size_t>(p.nodes) * 2 * sizeof(double) <= kTreeSmemLimit;
@@ -159,6 +163,8 @@ __device__ __forceinline__ bool beats(float v_other, int i_other, float v_me, in
 
 __global__ void __launch_bounds__(kTreeThreads)
 prune_kernel(const PruneLaunch p) {
+    pdl_release();
+    pdl_wait();
     extern __shared__ unsigned char keep[];            // per node, then (small trees) the node values as floats
     const int tree = blockIdx.x;
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
@@ -236,6 +242,8 @@ prune_kernel(const PruneLaunch p) {
 // Clipped GRPO objective (Eq. 5), forward value: one CTA per tree; per-thread strided sums, fixed-order reduction.
 __global__ void __launch_bounds__(kTreeThreads)
 objective_kernel(const ObjectiveLaunch p) {
+    pdl_release();
+    pdl_wait();
     const int tree = blockIdx.x;
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     double sum = 0.0;
@@ -271,8 +279,7 @@ objective_kernel(const ObjectiveLaunch p) {
 }  // namespace
 
 cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s) {
-    objective_kernel<<<p.n_trees, kTreeThreads, 0, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(objective_kernel, p.n_trees, kTreeThreads, 0, s, p);
 }
 
 cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s) {
@@ -282,8 +289,7 @@ cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s) {
         cudaError_t e = cudaFuncSetAttribute(fusion_ess_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
     }
-    fusion_ess_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(fusion_ess_kernel, p.n_trees, kTreeThreads, smem, s, p);
 }
 
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
@@ -293,8 +299,7 @@ cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
         cudaError_t e = cudaFuncSetAttribute(fuse_advantage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
     }
-    fuse_advantage_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(fuse_advantage_kernel, p.n_trees, kTreeThreads, smem, s, p);
 }
 
 cudaError_t launch_prune(const PruneLaunch& p0, cudaStream_t s) {
@@ -306,8 +311,7 @@ cudaError_t launch_prune(const PruneLaunch& p0, cudaStream_t s) {
         cudaError_t e = cudaFuncSetAttribute(prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
     }
-    prune_kernel<<<p.n_trees, kTreeThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(prune_kernel, p.n_trees, kTreeThreads, smem, s, p);
 }
 
 }  // namespace bgrpo

@@ -82,6 +82,8 @@ __device__ __forceinline__ double row_total(const double* partials, int64_t row,
 __global__ void __launch_bounds__(kStreamThreads)
 root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters, int32_t* status, int64_t D,
             int32_t n_trees, int32_t nodes_cap, int32_t nchunks, uint32_t node_id_base, const __grid_constant__ PhiloxKeys keys) {
+    pdl_release();
+    pdl_wait();           // the buffers may still be read by the kernels of the previous pass
     const int chunk = blockIdx.x % nchunks;
     const int tree = blockIdx.x / nchunks;
     const int64_t D4 = D >> 2;
@@ -282,6 +284,8 @@ step_kernel(const __grid_constant__ StepLaunch p) {
 // Flush: adds up a pending level outside a step launch (the tree is complete, or tree_logprob is done).
 __global__ void __launch_bounds__(kStreamThreads)
 finalize_kernel(const FinalizeDesc f, const float* partialsf, int32_t n_trees, int32_t nodes_cap, int32_t nchunks, int64_t D) {
+    pdl_release();
+    pdl_wait();
     finalize_rows(f, partialsf, n_trees, nodes_cap, nchunks, D, blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5),
                   gridDim.x * (kStreamThreads / 32));
 }
@@ -291,6 +295,8 @@ finalize_kernel(const FinalizeDesc f, const float* partialsf, int32_t n_trees, i
 template <int MODE>
 __global__ void __launch_bounds__(kStreamThreads)
 reward_kernel(const __grid_constant__ RewardLaunch p) {
+    pdl_release();
+    pdl_wait();
     const int chunk = blockIdx.x % p.nchunks;
     const int row = blockIdx.x / p.nchunks;             // tree * leaves + l
     const int tree = row / p.leaves;
@@ -363,11 +369,9 @@ cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t
 
 cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s) {
     const unsigned int grid = static_cast<unsigned int>(t->desc.n_trees) * t->nchunks;
-    root_kernel<<<grid, kStreamThreads, 0, s>>>(t->buf.latents, t->buf.node_table, t->buf.logp, t->counters, t->status, t->D,
-                                                t->desc.n_trees, t->desc.nodes_cap, t->nchunks,
-                                                static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap),
-                                                make_philox_keys(t->desc.seed));
-    return cudaGetLastError();
+    return launch_overlapped(root_kernel, grid, kStreamThreads, 0, s, t->buf.latents, t->buf.node_table, t->buf.logp, t->counters,
+                             t->status, t->D, t->desc.n_trees, t->desc.nodes_cap, t->nchunks,
+                             static_cast<uint32_t>(t->desc.tree_id_base * t->desc.nodes_cap), make_philox_keys(t->desc.seed));
 }
 
 cudaError_t launch_step(const StepLaunch& p, cudaStream_t s) {
@@ -386,16 +390,15 @@ cudaError_t launch_step(const StepLaunch& p, cudaStream_t s) {
 cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStream_t s) {
     const int rows = t->desc.n_trees * f.W;
     const int grid = (rows + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
-    finalize_kernel<<<grid < 1 ? 1 : grid, kStreamThreads, 0, s>>>(f, t->partialsf, t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D);
-    return cudaGetLastError();
+    return launch_overlapped(finalize_kernel, grid < 1 ? 1 : grid, kStreamThreads, 0, s, f, static_cast<const float*>(t->partialsf),
+                             t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D);
 }
 
 cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
     const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * p.nchunks;
     if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (p.mode == 0) reward_kernel<0><<<static_cast<unsigned int>(items), kStreamThreads, 0, s>>>(p);
-    else reward_kernel<1><<<static_cast<unsigned int>(items), kStreamThreads, 0, s>>>(p);
-    return cudaGetLastError();
+    if (p.mode == 0) return launch_overlapped(reward_kernel<0>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
+    return launch_overlapped(reward_kernel<1>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
 }
 
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {
