@@ -21,52 +21,6 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-// Publishes NV per-thread float sums of this CTA as doubles in partials[(row_b*nchunks + chunk)*3 + comp]
-// (row_b = row0 + v / comps) and takes a ticket on `counter`.  Only warp 0 returns with a meaningful value: true in
-// the CTA whose ticket was the row's last, after which every chunk partial of the row is visible to it.  The other
-// warps have nothing left to do once their sums are in shared memory.  Sums are float inside a warp (WARP_FLOAT:
-// 512 elements, a fixed shuffle tree) or double from the thread level on, and double across warps and chunks.
-template <int NV, bool WARP_FLOAT>
-__device__ __forceinline__ bool publish_partials(const float (&acc)[NV], double* partials, unsigned int* counter,
-                                                 int64_t row0, int comps, int nchunks, int chunk) {
-    __shared__ double red[NV][kWarps];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        double s;
-        if (WARP_FLOAT) {
-            float f = acc[v];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) f += __shfl_down_sync(0xffffffffu, f, o);
-            s = static_cast<double>(f);
-        } else {
-            s = warp_sum(static_cast<double>(acc[v]));
-        }
-        if (lane == 0) red[v][warp] = s;
-    }
-    __syncthreads();
-    if (warp != 0) return false;
-    int last = 0;
-    if (lane == 0) {
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            double s = 0.0;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) s += red[v][w];
-            const int64_t row = row0 + v / comps;
-            __stcg(&partials[(row * nchunks + chunk) * kPartialStride + (v % comps)], s);
-        }
-        __threadfence();
-        const unsigned int ticket = atomicAdd(counter, 1u);
-        last = (ticket == static_cast<unsigned int>(nchunks) - 1u);
-        if (last) {
-            *counter = 0u;        // every CTA of the row has arrived: leave the counter ready for the next launch
-            __threadfence();
-        }
-    }
-    return __shfl_sync(0xffffffffu, last, 0) != 0;
-}
-
 // Sum of one component of a row's chunk partials, in chunk order within each lane and a fixed shuffle tree across
 // lanes.  Called by whole warps only.
 __device__ __forceinline__ double row_total(const double* partials, int64_t row, int comp, int nchunks) {
@@ -335,16 +289,42 @@ reward_kernel(const __grid_constant__ RewardLaunch p) {
             }
         }
     }
-    const bool last = publish_partials<NV, false>(acc, p.partials, &p.counters[node_row], node_row, NV, p.nchunks, chunk);
-    if (!last) return;                                  // only warp 0 of the row's last CTA goes on
+    // One double per (row, chunk, component): thread sums are float over 16 elements, double from the warp level on.
+    // Nothing waits for these stores; reward_finish_kernel, next on the stream, adds the chunks up in order.
+    __shared__ double red[NV][kWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const double s = warp_sum(static_cast<double>(acc[v]));
+        if (lane == 0) red[v][warp] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < NV) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
+        p.partials[(node_row * p.nchunks + chunk) * kPartialStride + threadIdx.x] = s;
+    }
+}
+
+// One warp per leaf row: the row's chunk partials in chunk order within each lane, a fixed shuffle tree across lanes.
+template <int MODE>
+__global__ void __launch_bounds__(kStreamThreads)
+reward_finish_kernel(const __grid_constant__ RewardLaunch p) {
+    pdl_release();
+    pdl_wait();
+    const int row = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5);      // tree * leaves + l
+    if (row >= p.n_trees * p.leaves) return;
+    const int tree = row / p.leaves;
+    const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + (row - tree * p.leaves);
     if (MODE == 0) {
         const double ss = row_total(p.partials, node_row, 0, p.nchunks);
-        if (threadIdx.x == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
+        if ((threadIdx.x & 31) == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
     } else {
         const double dot = row_total(p.partials, node_row, 0, p.nchunks);
         const double zz = row_total(p.partials, node_row, 1, p.nchunks);
         const double tt = row_total(p.partials, node_row, 2, p.nchunks);
-        if (threadIdx.x == 0)
+        if ((threadIdx.x & 31) == 0)
             p.r[row] = static_cast<float>(static_cast<double>(p.r[row]) + static_cast<double>(p.scale) * dot / (sqrt(zz) * sqrt(tt)));
     }
 }
@@ -397,8 +377,17 @@ cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStre
 cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
     const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * p.nchunks;
     if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (p.mode == 0) return launch_overlapped(reward_kernel<0>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
-    return launch_overlapped(reward_kernel<1>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
+    const unsigned int rows = static_cast<unsigned int>(p.n_trees) * static_cast<unsigned int>(p.leaves);
+    const unsigned int fgrid = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
+    cudaError_t e;
+    if (p.mode == 0) {
+        e = launch_overlapped(reward_kernel<0>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
+        if (e == cudaSuccess) e = launch_overlapped(reward_finish_kernel<0>, fgrid, kStreamThreads, 0, s, p);
+    } else {
+        e = launch_overlapped(reward_kernel<1>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
+        if (e == cudaSuccess) e = launch_overlapped(reward_finish_kernel<1>, fgrid, kStreamThreads, 0, s, p);
+    }
+    return e;
 }
 
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {

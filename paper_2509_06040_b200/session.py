@@ -134,6 +134,6 @@ class TreeSession:
             n = 1 + 2                                              # root + whole-tree rollout + its log-prob sums
         else:
             n = 1 + w.T * (2 if w.velocity == "mlp" else 1) + 1   # root + (mlp +) step per depth + log-prob flush
-        n += 1 if w.reward in ("neg_mse_mu", "neg_mse_target", "normal_plus_cos") else 0
+        n += 2 if w.reward in ("neg_mse_mu", "neg_mse_target", "normal_plus_cos") else 0   # partial sums + their fixed-order total
         n += 2                                                     # fuse+advantage, prune
         return n
