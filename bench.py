@@ -43,8 +43,8 @@ NOMINAL_HBM_GBS = 8000.0
 # reported per launch is bytes-per-unit times the units of an average launch of the timed workload (traffic grows in
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
-    "step_kernel": {"workload": "video", "bytes": 75.589888e6 + 15.569152e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "8edf0b481da5"},
+    "step_kernel": {"workload": "video", "bytes": 75.599616e6 + 12.611840e6, "units": 8 * 2096640,
+                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "8465fe6dcf94"},
     "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.295808e6 + 214.387712e6, "units": 1036800,
                             "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "2141aa3f7a6b"},
     "rollout_fused_kernel": {"workload": "video", "bytes": 16.817152e6 + 866.026752e6, "units": 110 * 2096640,
