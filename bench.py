@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
     "step_kernel": {"workload": "video", "bytes": 75.599616e6 + 12.611840e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "8465fe6dcf94"},
+                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "0f5299a50f5b"},
     "mlp_velocity_kernel": {"workload": "image_batch", "bytes": 266.295808e6 + 214.387712e6, "units": 1036800,
                             "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "2141aa3f7a6b"},
     "rollout_fused_kernel": {"workload": "video", "bytes": 16.817152e6 + 866.026752e6, "units": 110 * 2096640,

@@ -17,7 +17,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbgrpo.so")
-SOURCES = ["api.cu", "tree_step.cu", "tree_fused.cu", "tree_reduce.cu", "mlp_velocity.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "tree_step.cu", "tree_reward.cu", "tree_fused.cu", "tree_reduce.cu", "mlp_velocity.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -1,6 +1,5 @@
 // Streaming kernels of the rollout: root initialisation, the fused gather / fork / Euler-Maruyama update /
-// log-prob step (Eq. 2 and the appendix's Euler-Maruyama form), the log-prob recompute under a given velocity,
-// and the leaf-reward reductions.  All of them are HBM-bound: every latent element is read or written once,
+// log-prob step (Eq. 2 and the appendix's Euler-Maruyama form) and the log-prob recompute under a given velocity.  All of them are HBM-bound: every latent element is read or written once,
 // with 128-bit accesses, and the noise is generated in registers.
 //
 // Sums over a row are float32 inside a thread (inside a warp for the step's log-prob), double from there on, and
@@ -13,22 +12,11 @@ namespace {
 
 constexpr int kVecPerThread = kChunkVec / kStreamThreads;   // 4
 constexpr int kWarps = kStreamThreads / 32;
-constexpr int kPartialStride = 3;                           // doubles per (row, chunk) slot
 
 __device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
     return x;
-}
-
-// Sum of one component of a row's chunk partials, in chunk order within each lane and a fixed shuffle tree across
-// lanes.  Called by whole warps only.
-__device__ __forceinline__ double row_total(const double* partials, int64_t row, int comp, int nchunks) {
-    const int lane = threadIdx.x & 31;
-    double s = 0.0;
-    for (int c = lane; c < nchunks; c += 32) s += __ldcg(&partials[(row * nchunks + c) * kPartialStride + comp]);
-    s = warp_sum(s);
-    return __shfl_sync(0xffffffffu, s, 0);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -244,91 +232,6 @@ finalize_kernel(const FinalizeDesc f, const float* partialsf, int32_t n_trees, i
                   gridDim.x * (kStreamThreads / 32));
 }
 
-// ---------------------------------------------------------------------------------------------------------------
-// Leaf rewards: mode 0  r = -mean (z - target)^2 ; mode 1  r += scale * cos(z, target).
-template <int MODE>
-__global__ void __launch_bounds__(kStreamThreads)
-reward_kernel(const __grid_constant__ RewardLaunch p) {
-    pdl_release();
-    pdl_wait();
-    const int chunk = blockIdx.x % p.nchunks;
-    const int row = blockIdx.x / p.nchunks;             // tree * leaves + l
-    const int tree = row / p.leaves;
-    const int l = row - tree * p.leaves;
-    const int64_t D4 = p.D >> 2;
-    const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + l;
-    const float4* __restrict__ z = reinterpret_cast<const float4*>(p.latents + node_row * p.D);
-    const float4* __restrict__ tg = reinterpret_cast<const float4*>(p.target + static_cast<int64_t>(tree) * p.D);
-    constexpr int NV = (MODE == 0) ? 1 : 3;
-    float acc[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) acc[v] = 0.0f;
-    const int64_t e0 = static_cast<int64_t>(chunk) * kChunkVec + threadIdx.x;
-    float4 a[kVecPerThread], t[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int64_t e = e0 + k * kStreamThreads;
-        if (e < D4) { a[k] = __ldcs(z + e); t[k] = __ldg(tg + e); }
-    }
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int64_t e = e0 + k * kStreamThreads;
-        if (e < D4) {
-            const float av[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
-            const float tv[4] = {t[k].x, t[k].y, t[k].z, t[k].w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (MODE == 0) {
-                    const float d = av[q] - tv[q];
-                    acc[0] = fmaf(d, d, acc[0]);
-                } else {
-                    acc[0] = fmaf(av[q], tv[q], acc[0]);
-                    acc[1] = fmaf(av[q], av[q], acc[1]);
-                    acc[2] = fmaf(tv[q], tv[q], acc[2]);
-                }
-            }
-        }
-    }
-    // One double per (row, chunk, component): thread sums are float over 16 elements, double from the warp level on.
-    // Nothing waits for these stores; reward_finish_kernel, next on the stream, adds the chunks up in order.
-    __shared__ double red[NV][kWarps];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const double s = warp_sum(static_cast<double>(acc[v]));
-        if (lane == 0) red[v][warp] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x < NV) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
-        p.partials[(node_row * p.nchunks + chunk) * kPartialStride + threadIdx.x] = s;
-    }
-}
-
-// One warp per leaf row: the row's chunk partials in chunk order within each lane, a fixed shuffle tree across lanes.
-template <int MODE>
-__global__ void __launch_bounds__(kStreamThreads)
-reward_finish_kernel(const __grid_constant__ RewardLaunch p) {
-    pdl_release();
-    pdl_wait();
-    const int row = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5);      // tree * leaves + l
-    if (row >= p.n_trees * p.leaves) return;
-    const int tree = row / p.leaves;
-    const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + (row - tree * p.leaves);
-    if (MODE == 0) {
-        const double ss = row_total(p.partials, node_row, 0, p.nchunks);
-        if ((threadIdx.x & 31) == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));
-    } else {
-        const double dot = row_total(p.partials, node_row, 0, p.nchunks);
-        const double zz = row_total(p.partials, node_row, 1, p.nchunks);
-        const double tt = row_total(p.partials, node_row, 2, p.nchunks);
-        if ((threadIdx.x & 31) == 0)
-            p.r[row] = static_cast<float>(static_cast<double>(p.r[row]) + static_cast<double>(p.scale) * dot / (sqrt(zz) * sqrt(tt)));
-    }
-}
-
 __global__ void philox_words_kernel(const __grid_constant__ PhiloxKeys keys, uint32_t node, uint32_t step, uint32_t tag, uint4* out, int64_t nblk) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i < nblk) out[i] = philox4x32_10(make_uint4(static_cast<uint32_t>(i), node, step, tag), keys);
@@ -372,22 +275,6 @@ cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStre
     const int grid = (rows + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
     return launch_overlapped(finalize_kernel, grid < 1 ? 1 : grid, kStreamThreads, 0, s, f, static_cast<const float*>(t->partialsf),
                              t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D);
-}
-
-cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
-    const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * p.nchunks;
-    if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    const unsigned int rows = static_cast<unsigned int>(p.n_trees) * static_cast<unsigned int>(p.leaves);
-    const unsigned int fgrid = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
-    cudaError_t e;
-    if (p.mode == 0) {
-        e = launch_overlapped(reward_kernel<0>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
-        if (e == cudaSuccess) e = launch_overlapped(reward_finish_kernel<0>, fgrid, kStreamThreads, 0, s, p);
-    } else {
-        e = launch_overlapped(reward_kernel<1>, static_cast<unsigned int>(items), kStreamThreads, 0, s, p);
-        if (e == cudaSuccess) e = launch_overlapped(reward_finish_kernel<1>, fgrid, kStreamThreads, 0, s, p);
-    }
-    return e;
 }
 
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {
