@@ -400,6 +400,38 @@ def fused_rollout_line(w, device, peaks, reps):
     return out
 
 
+def savings_line(w, s_tree, device, reps):
+    """The tree against an equal-leaf-count batch of independent sequential rollouts through the same kernels
+    (K = 1, no split, n_trees x leaves trees of T steps): model evaluations and measured rollout time."""
+    import torch
+    from paper_2509_06040_b200.session import TreeSession
+
+    def rollout_ms(sess, ww):
+        for k in range(2):
+            sess.rollout(seed=ww.seed + 5000 + k)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for k in range(reps):
+            sess.rollout(seed=ww.seed + 5100 + k)
+        a1.record()
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) / reps
+
+    t_tree = rollout_ms(s_tree, w)
+    wseq = w.scaled(name=w.name + "_sequential", n_trees=w.n_trees * w.leaves, K=1, splits=())
+    seq = TreeSession(wseq, device=device)
+    seq.upload_inputs(make_inputs(wseq))
+    t_seq = rollout_ms(seq, wseq)
+    del seq
+    torch.cuda.empty_cache()
+    return {"leaves": w.n_trees * w.leaves, "model_evals_tree": w.n_trees * w.model_evals,
+            "model_evals_sequential": w.n_trees * w.leaves * w.T,
+            "model_evals_ratio": (w.leaves * w.T) / w.model_evals,
+            "rollout_ms_tree": t_tree, "rollout_ms_sequential": t_seq, "rollout_time_ratio": t_seq / t_tree,
+            "note": "sequential = the same number of final samples as independent T-step rollouts (K = 1) through the same kernels"}
+
+
 # ------------------------------------------------------------------------------------------------ GPU arm
 def run_ours(args, w):
     import torch
@@ -575,6 +607,11 @@ def run_ours(args, w):
             if w2.velocity == "linear":
                 also[name]["fused_rollout"] = fused_rollout_line(w2, f"cuda:{local}", peaks, n2)
 
+    # ---- the tree against independent sequential rollouts with as many final samples (rank 0, single GPU)
+    savings = None
+    if rank == 0 and world == 1 and not args.no_also:
+        savings = savings_line(w, s, f"cuda:{local}", max(3, min(10, args.steps)))
+
     # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -601,7 +638,7 @@ def run_ours(args, w):
                             "pass k computes; results of every pass copied back to pinned host memory",
                     "one_pass_at_a_time": e2e_serial},
             "gpu_launches": s.kernel_launches_per_pass() * args.steps,
-            "clocks": clocks, "kernel_ms_per_pass": breakdown, "also": also,
+            "clocks": clocks, "kernel_ms_per_pass": breakdown, "savings": savings, "also": also,
         }
         if roof is not roof_step:
             line["roofline_step"] = roof_step
