@@ -153,3 +153,87 @@ def test_step_kernel_full_size_sampled_rows(B, name, depth):
     tab = s.node_table.cpu().numpy().reshape(4, w.n_trees, s.nodes_cap)
     assert np.array_equal(tab[0, 0, off_c:off_c + W * fan], off + np.arange(W * fan) // fan)
     assert np.all(tab[1, :, off_c:off_c + W * fan] == depth + 1)
+
+
+def test_cosine_reward_at_the_image_size_every_row(B):
+    """The cosine leaf reward of the 32-tree image batch in the launch configuration the benchmark times: 512 leaf rows
+    of 129 600 elements (32 chunks of 4096 per row, exactly one lane-stride of the finish kernel's sum) filled with
+    seeded normals, every row against the oracle (Algorithm 1, "Evaluate rewards for leaves")."""
+    from paper_2509_06040_b200.session import TreeSession
+    w = CONFIGS["image_batch"]
+    inp = make_inputs(w)
+    s = TreeSession(w)
+    s.upload_inputs(inp)
+    s.init()
+    s.v.zero_()
+    for i in range(w.T):                          # grow the tree; the leaf rows are replaced below
+        B.tree_step(s.tree, 1 if i in w.splits else 0, s.v)
+    widths, offs = B.tree_levels(s.tree)
+    L, off = widths[w.T], offs[w.T]
+    assert L == w.leaves == 16
+    rng = np.random.default_rng([13, w.n_trees])
+    z = (0.7 * rng.standard_normal((w.n_trees, L, w.D), dtype=np.float32) + 0.05 * inp.target[:, None, :]).astype(np.float32)
+    s.latents[:, off:off + L].copy_(torch.from_numpy(z))
+    s.rewards()                                   # seeded draw + 0.1 cos(z_leaf, target)
+    first = s.leaf_r.clone()
+    s.rewards()
+    torch.cuda.synchronize()
+    B.tree_sync_status(s.tree)
+    assert torch.equal(first, s.leaf_r)           # fixed summation order: the same bits on a second run
+    got = s.leaf_r.cpu().numpy()
+    worst = 0.0
+    for t in range(w.n_trees):
+        for q in range(L):
+            ref = float(inp.reward_draws[t, q]) + 0.1 * rewards.cosine(z[t, q], inp.target[t])
+            worst = max(worst, abs(got[t, q] - ref) / max(1.0, abs(ref)))
+    assert worst <= 1e-6, worst
+    # and the -MSE mode on the same rows
+    B.leaf_reward_mse(s.tree, s.target, s.leaf_r)
+    torch.cuda.synchronize()
+    got = s.leaf_r.cpu().numpy()
+    for t in range(w.n_trees):
+        for q in range(L):
+            ref = rewards.neg_mse(z[t, q], inp.target[t])
+            assert abs(got[t, q] - ref) <= 1e-6 * max(1.0, abs(ref))
+
+
+@pytest.mark.parametrize("name", ["image_batch", "group"])
+def test_reductions_with_the_batched_configs_tree_counts(B, name):
+    """Reward fusion, depth-wise advantages and the pruning masks launched as the batched configurations launch them -
+    32 trees with top-2 per split and the seeded 4 of 16 pruned steps; 8 trees of 765 nodes with the mixture rewards -
+    every tree against the oracle (Eq. 3, Eq. 4, "Pruning Strategies").  The reductions never look at the latents, so
+    the trees are grown with 16 elements per node; rewards and log-probs are teacher-forced in float32."""
+    from paper_2509_06040_b200.session import TreeSession
+    cfg = CONFIGS[name]
+    inp_full = make_inputs(cfg.scaled(tokens=1, channels=64))       # the per-leaf reward draws and pruned steps of the config
+    w = cfg.scaled(name=name + "_reductions", tokens=4, channels=4, velocity="linear", reward="neg_mse_mu")
+    s = TreeSession(w)
+    s.upload_inputs(make_inputs(w))
+    s.rollout()
+    s.pruned_steps = tuple(int(x) for x in inp_full.pruned_steps)
+    topo = otree.build_topology(w.T, w.K, w.splits)
+    assert topo.nodes == cfg.nodes
+    rng = np.random.default_rng([17, w.n_trees])
+    r = inp_full.reward_draws.astype(np.float32)
+    lp = (-0.9 + 0.2 * rng.standard_normal((w.n_trees, topo.nodes))).astype(np.float32)
+    lp[:, 0] = 0
+    s.logp.copy_(torch.from_numpy(lp))
+    s.leaf_r.copy_(torch.from_numpy(r))
+    for beta in (w.beta, 1.0):
+        B.tree_fuse_advantage(s.tree, s.leaf_r, beta, 1.0, f32(w.eps), f32(w.adv_clip))
+        s.prune()
+        torch.cuda.synchronize()
+        B.tree_sync_status(s.tree)
+        got_rbar, got_adv, got_mask = s.rbar.cpu().numpy(), s.adv.cpu().numpy(), s.mask.cpu().numpy()
+        for t in range(w.n_trees):
+            rbar = credit.fuse_rewards(topo, r[t].astype(np.float64), lp[t].astype(np.float64), beta)
+            adv = credit.depth_advantages(topo, rbar, f32(w.eps))
+            assert np.abs(got_rbar[t] - rbar).max() <= 1e-6 * max(1.0, np.abs(rbar).max()), t
+            assert adv_close(got_adv[t], adv), t
+            mask = credit.gradient_mask(topo, got_rbar[t], w.width_mode, w.width_k, s.pruned_steps, w.ignore_last_step)
+            assert np.array_equal(got_mask[t], mask), t
+    if name == "image_batch":
+        assert len(s.pruned_steps) == 4
+        # top-2 of 2 children keeps every child: the mask is exactly the depth mask (reading R8 of the configs)
+        depth_only = credit.gradient_mask(topo, got_rbar[0], 0, 0, s.pruned_steps, False)
+        assert np.array_equal(got_mask[0], depth_only)

@@ -266,13 +266,16 @@ def test_logprob_all_edges_linear_velocity(B):
     torch.cuda.synchronize()
     grid = w.t_grid().astype(np.float64)
     got = out.cpu().numpy()
+    worst = 0.0
     for t in range(2):
         mu_h = (inp.mu[t] + np.float32(0.1)).astype(np.float64)
         for c in range(1, topo.nodes):
             p, i = int(topo.parent[c]), int(topo.depth[c]) - 1
             v = sde.linear_velocity(lat[t][p].astype(np.float64), grid[i], mu_h, 0.5)
             ref = sde.edge_logp(lat[t][p], lat[t][c], v, grid[i], grid[i] - grid[i + 1], f32(w.sigma))
-            assert abs(got[t, c] - ref) <= 2e-5 * max(1.0, abs(ref))
+            worst = max(worst, abs(got[t, c] - ref))
+    print("worst |logp - oracle| under the perturbed policy:", worst)
+    assert worst <= LOGP_TOL, worst
 
 
 # ---------------------------------------------------------------------------------------------- rewards

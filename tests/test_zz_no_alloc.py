@@ -1,9 +1,9 @@
 """bgrpo_reward_mse_static: the leaf-reward reduction for callers that cannot allocate device memory where they
 call the library (all memory already given to their own pool, or a cudaMalloc there would stall the whole device).
 It keeps its reduction scratch in an array built into the library, so this test checks, through the C ABI, that it
-returns what the ordinary entry point (bgrpo_leaf_reward_mse, caller-allocated scratch) returns - on two calls in a
-row with different shapes, because the built-in array is shared by all calls and keeps the previous call's contents -
-and that sizes beyond the built-in array are refused.  The file name makes pytest collect it last."""
+returns what the ordinary entry point (bgrpo_leaf_reward_mse, caller-allocated scratch) returns and what the CPU oracle
+computes from the same rows - on several calls in a row with different shapes, because the built-in array is shared by
+all calls and keeps the previous call's contents - and that sizes beyond the built-in array are refused.  The file name makes pytest collect it last."""
 import numpy as np
 import pytest
 import torch
@@ -36,16 +36,20 @@ def _leaf_rewards_both_ways(B, tokens, K, splits, seed):
     out = torch.full((leaves,), float("nan"), device="cuda")
     B.reward_mse_static(rows, s.target[0], leaves, w.D, out)
     torch.cuda.synchronize()
-    return s.leaf_r[0].cpu().numpy(), out.cpu().numpy()
+    from oracle import rewards
+    rows_h, target_h = rows.cpu().numpy(), s.target[0].cpu().numpy()
+    oracle = np.array([rewards.neg_mse(rows_h[i], target_h) for i in range(leaves)])
+    return s.leaf_r[0].cpu().numpy(), out.cpu().numpy(), oracle
 
 
 def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row(B):
     # first call: 9 rows of 3 chunks with a ragged tail; second call: 4 rows of 1 chunk - fewer rows and chunks
     # than the call before, so stale partials and counters from the first call sit right beside the live ones
     for tokens, K, splits, seed in ((2125, 3, (0, 2), 5), (300, 2, (0, 1), 6), (2125, 3, (0, 2), 7)):
-        ref, got = _leaf_rewards_both_ways(B, tokens, K, splits, seed)
+        ref, got, oracle = _leaf_rewards_both_ways(B, tokens, K, splits, seed)
         assert np.all(np.isfinite(got))
         assert np.abs(got - ref).max() <= 1e-6 * max(1.0, np.abs(ref).max())
+        assert np.abs(got - oracle).max() <= 1e-6 * max(1.0, np.abs(oracle).max())
 
 
 def test_sizes_beyond_the_built_in_array_are_refused(B):
