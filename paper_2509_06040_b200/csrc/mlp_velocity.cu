@@ -34,7 +34,7 @@
 // takes 1/S of the chunks and writes its partial output tile to scratch; the CTA that draws the tile's last ticket adds the
 // S partials in part order and writes v, so the result does not depend on which CTA finishes first.
 //
-// Every wait is bounded (2 s): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
+// Every wait is bounded (about 2 s of SM clock): on a timeout the thread raises the abort flag, all roles drain, tensor memory is
 // released and bit 2 of the status word is set.
 #include "internal.h"
 
@@ -56,7 +56,7 @@ constexpr uint32_t kTmemCols = 512;       // D1: 2 x 128 columns, H: 2 x 64, D2:
 constexpr uint32_t kHCol = 2 * kHc;
 constexpr uint32_t kD2Col = kHCol + 2 * (kHc / 2);
 constexpr int kGroupWarps = kEpiWarps / 2; // epilogue warps that work on one chunk
-constexpr unsigned long long kWaitNs = 2000000000ull;
+constexpr long long kWaitCycles = 4000000000ll;      // about two seconds of SM clock
 
 struct MlpSmem {
     alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
@@ -93,10 +93,14 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
 __device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase of the given parity; false after kWaitNs or once another thread has raised the abort flag.
+// Bounded wait for the phase of the given parity; false once kWaitCycles have passed or another thread has raised the
+// abort flag.  The loop is nothing but the hardware's own try_wait (which parks the thread until the phase completes or
+// its internal time slice ends): the clock and the abort flag are looked at once every 64 polls, so a handoff between
+// two roles costs the barrier's latency and not a poll of timers and flags on top.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort_flag) {
     const uint32_t addr = smem_u32(bar);
-    {   // common case: the phase is already complete, or completes within the hardware's own suspend window
+    long long t0 = 0;
+    for (uint32_t polls = 1;; ++polls) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -104,21 +108,12 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
-    }
-    unsigned long long t0 = 0;
-    for (;;) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-        if (*abort_flag) return false;
-        unsigned long long now;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > kWaitNs) { *abort_flag = 1; return false; }
+        if ((polls & 63u) == 0u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+        }
     }
 }
 // True in exactly one lane of a converged warp.  Code guarded by it is known to the compiler to run in a single
@@ -593,71 +588,64 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             return true;
         };
         // 32 accumulator columns -> 16 registers of packed bf16 activation pairs
-        // The packed polynomial covers |x| < 2; the OR of the packed inputs shows whether any of this thread's 32 values
-        // lies outside (its top exponent bit is set), and only then the thread redoes its values with the hardware tanh.
-        // With weights and latents of the usual scale (pre-activations of standard deviation ~0.2) that never happens.
-        auto activate = [&](const uint32_t (&acc)[32], uint32_t (&pk)[16]) {
+        // One chunk of this warp: 64 accumulator columns arrive as float32, are rounded to packed bf16 pairs at once (32
+        // registers) and D1 is handed back before any arithmetic, so GEMM1 of chunk g + 2 runs under the activation of
+        // chunk g.  The packed polynomial covers |x| < 2; the OR of the packed inputs shows whether any of this thread's
+        // 64 values lies outside (its top exponent bit is set), and only then the thread takes the hardware-tanh form
+        // for its values.  With weights and latents of the usual scale (pre-activations of standard deviation ~0.2) that
+        // never happens.
+        auto pack16 = [&](const uint32_t (&acc)[32], uint32_t* xb) {
+#pragma unroll
+            for (int m = 0; m < 16; ++m) xb[m] = pack_bf16(__uint_as_float(acc[2 * m]), __uint_as_float(acc[2 * m + 1]));
+        };
+        auto activate = [&](uint32_t (&xb)[32]) {
             uint32_t seen = 0u;
 #pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                const uint32_t xb = pack_bf16(__uint_as_float(acc[2 * m]), __uint_as_float(acc[2 * m + 1]));
-                seen |= xb;
-                pk[m] = gelu_x2_poly(xb);
-            }
-            if (seen & kGeluRangeBits) {
+            for (int m = 0; m < 32; ++m) seen |= xb[m];
+            if (!(seen & kGeluRangeBits)) {
 #pragma unroll
-                for (int m = 0; m < 16; ++m)
-                    pk[m] = pack_bf16(gelu_x2(__uint_as_float(acc[2 * m])), gelu_x2(__uint_as_float(acc[2 * m + 1])));
+                for (int m = 0; m < 32; ++m) xb[m] = gelu_x2_poly(xb[m]);
+            } else {
+#pragma unroll
+                for (int m = 0; m < 32; ++m)
+                    xb[m] = pack_bf16(gelu_x2(__uint_as_float(xb[m] << 16)), gelu_x2(__uint_as_float(xb[m] & 0xffff0000u)));
             }
         };
         const uint32_t d1_slice = tmem + lane_addr + static_cast<uint32_t>(group) * kHc + (sub & 1u) * 64u;              // 64 fp32 columns
         const uint32_t h_slice = tmem + lane_addr + kHCol + static_cast<uint32_t>(group) * (kHc / 2) + (sub & 1u) * 32u;  // 32 packed columns
 
-        uint32_t acc[32], pk[16];
+        uint32_t acc[32], xb[32];
         int g = group;                // chunk index within this CTA's sequence of tiles x chunks; use number g >> 1 of the buffers
-        if (g < n_my_chunks) {        // first 32 columns of the first chunk
+        if (g < n_my_chunks)
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], 0u, abort_flag) ? 1 : 0) != 0;
-            if (ok) {
-                tc_fence_after();
-                tmem_ld32(d1_slice, acc);
-                tmem_ld_wait32(acc);
-            }
-        }
         for (; g < n_my_chunks && ok; g += 2) {
             // tiles whose last GEMM2 was issued at least two chunks ago
             while (ok && (next_out + 1) * NC + 2 <= g) ok = output_tile(next_out++);
             if (!ok) break;
             const uint32_t use = static_cast<uint32_t>(g >> 1);
-            // is the GEMM2 that read this group's previous activations done?  (asked now, needed after the arithmetic)
-            uint32_t h_ready = 1u;
-            if (g >= 2) h_ready = mbar_probe(&sm.h_free[group], (use - 1u) & 1u);
-            activate(acc, pk);                                // columns 0..31 of this warp's 64
-            tmem_ld32(d1_slice + 32u, acc);                   // columns 32..63, in flight during the store below
-            if (!__all_sync(0xffffffffu, h_ready))
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.h_free[group], (use - 1u) & 1u, abort_flag) ? 1 : 0) != 0;
-            if (ok) {
-                tc_fence_after();
-                tmem_st16(h_slice, pk);
-            }
+            tc_fence_after();
+            tmem_ld32(d1_slice, acc);
             tmem_ld_wait32(acc);
+            pack16(acc, xb);
+            tmem_ld32(d1_slice + 32u, acc);
+            tmem_ld_wait32(acc);
+            pack16(acc, xb + 16);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.d1_empty[group]);  // D1 of this chunk is in registers: GEMM1 of chunk g + 2 may go
+            activate(xb);
+            if (g >= 2)       // the GEMM2 that read this group's previous activations must be done before they are overwritten
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.h_free[group], (use - 1u) & 1u, abort_flag) ? 1 : 0) != 0;
             if (!ok) break;
-            activate(acc, pk);
-            tmem_st16(h_slice + 16u, pk);
+            tc_fence_after();
+            tmem_st16(h_slice, reinterpret_cast<const uint32_t (&)[16]>(xb[0]));
+            tmem_st16(h_slice + 16u, reinterpret_cast<const uint32_t (&)[16]>(xb[16]));
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.h_full[group]);
-            if (g + 2 < n_my_chunks) {                        // first half of the next chunk
+            if (g + 2 < n_my_chunks)
                 ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], (use + 1u) & 1u, abort_flag) ? 1 : 0) != 0;
-                if (ok) {
-                    tc_fence_after();
-                    tmem_ld32(d1_slice, acc);
-                    tmem_ld_wait32(acc);
-                }
-            }
         }
         while (ok && next_out < n_my_tiles) ok = output_tile(next_out++);
         tmem_ld_wait();
