@@ -57,6 +57,7 @@ constexpr uint32_t kHCol = 2 * kHc;
 constexpr uint32_t kD2Col = kHCol + 2 * (kHc / 2);
 constexpr int kGroupWarps = kEpiWarps / 2; // epilogue warps that work on one chunk
 constexpr long long kWaitCycles = 4000000000ll;      // about two seconds of SM clock
+constexpr uint32_t kSuspendHintNs = 20000u;            // how long one try_wait may park the thread before it reports "not yet"
 
 struct MlpSmem {
     alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
@@ -104,9 +105,9 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
         if (done) return true;
         if ((polls & 63u) == 0u) {
             if (*abort_flag) return false;
