@@ -5,23 +5,24 @@
 //
 // One persistent CTA per SM walks 128-token tiles.  For each tile the hidden dimension is cut into chunks of 128:
 //     GEMM1(c): D1[128 tok][128 hid]  = A[128 tok][64]      * W1_c        (4 MMAs of K = 16, accumulator in TMEM)
-//     GELU     : H_c = bf16(2 GELU(D1))  TMEM -> registers -> TMEM (64 columns of packed bf16 pairs): the hidden
-//                activation never leaves tensor memory
+//     GELU     : H_c = bf16(2 GELU(D1))  TMEM -> registers -> TMEM: the hidden activation never leaves tensor memory
 //     GEMM2(c): D2[128 tok][64]      += H_c[128 tok][128]   * W2_c        (8 MMAs of K = 16, A operand read from TMEM)
 // and the output tile is v = 0.5 D2 (the factor 1/2 of GELU is a power of two: taking it out of the 3072 activations
 // of a token and applying it to the 64 outputs changes no rounding).
+// Tensor memory (512 columns): three chunk buffers of 128 columns and two output accumulators of 64.  A chunk buffer
+// holds D1 of its chunk and then, in place, the packed activations: a warp reads its 64 accumulator columns into
+// registers and later writes its 32 packed columns over the first half of exactly those columns, so no warp ever writes
+// what another still has to read.  The buffer is free again when GEMM2 of the chunk has completed.  Three buffers for two
+// epilogue groups mean that GEMM1 of chunk c + 2 does not wait for the group that works on chunk c, and the group does
+// not wait for GEMM2 of chunk c - 2: the roles only meet at "accumulator ready" and "activations ready".
 // Warp roles:
 //     warp 0       streams the packed weights with bulk asynchronous copies: lane 0 feeds a 3-stage ring of W1 chunks,
 //                  lane 1 a 4-stage ring of W2 chunks;
-//     warp 1       owns tensor memory and issues GEMM1; D1 has one buffer per chunk parity, free again as soon as the
-//                  epilogue group of that parity has loaded it, so GEMM1(c + 2) runs during the epilogue of chunk c;
-//     warp 19      issues GEMM2 from the activation buffer of the chunk's parity;
+//     warp 1       owns tensor memory and issues GEMM1 into the buffer of the chunk (chunk index mod 3);
+//     warp 19      issues GEMM2 from the same buffer once the chunk's activations are in it;
 //     warps 2..17  GELU epilogue in two groups of eight: group p takes the chunks of parity p, two warps per TMEM lane
-//                  quarter with 64 columns each.  The groups run half a period apart, so one group's
-//                  arithmetic fills the issue slots while the other hands a chunk over (barrier round trips, TMEM
-//                  load latency); a warp issues the TMEM load of its NEXT chunk before it hands the current one to
-//                  GEMM2.  All sixteen warps write the output tile (D2 is double-buffered, and a tile is written out
-//                  two chunks after its last GEMM2 was issued, when it has long completed);
+//                  quarter with 64 columns each.  All sixteen warps write the output tile (D2 is double-buffered, and a
+//                  tile is written out two chunks after its last GEMM2 was issued, when it has long completed);
 //     warp 18      brings the NEXT tile's latents in with bulk asynchronous copies (one per tree the tile touches) into
 //                  a float32 staging buffer and converts them to the bf16 A tile while the current tile computes.  (Plain
 //                  loads from one warp kept only 4 KiB in flight and took longer per tile than the arithmetic.)  The
@@ -52,12 +53,11 @@ constexpr int kGemm2Warp = 3 + kEpiWarps;
 constexpr int kMlpThreads = (4 + kEpiWarps) * 32;
 constexpr uint32_t kTileBytes = kTok * 128;              // one [128 rows][128 B] operand tile = 16 KiB
 constexpr uint32_t kChunkBytes = 2 * kTileBytes;         // packed weights of a chunk: W1_c (16 KiB) then W2_c (16 KiB)
-constexpr uint32_t kTmemCols = 512;       // D1: 2 x 128 columns, H: 2 x 64, D2: 2 x 64; index = chunk parity (D1, H) or tile parity (D2)
-constexpr uint32_t kHCol = 2 * kHc;
-constexpr uint32_t kD2Col = kHCol + 2 * (kHc / 2);
+constexpr uint32_t kTmemCols = 512;       // three chunk buffers of 128 columns (index = chunk mod 3), then D2: 2 x 64 (index = tile parity)
+constexpr int kBufs = 3;
+constexpr uint32_t kD2Col = kBufs * kHc;
 constexpr int kGroupWarps = kEpiWarps / 2; // epilogue warps that work on one chunk
 constexpr long long kWaitCycles = 4000000000ll;      // about two seconds of SM clock
-constexpr uint32_t kSuspendHintNs = 20000u;            // how long one try_wait may park the thread before it reports "not yet"
 
 struct MlpSmem {
     alignas(1024) unsigned char w1[kW1Stages][kTileBytes];  // W1_c tile [128 n = hidden][128 B = 64 channels]
@@ -65,7 +65,7 @@ struct MlpSmem {
     alignas(1024) unsigned char a[2][kTileBytes];           // bf16(z) tile [128 tok][128 B], double-buffered over tiles
     alignas(1024) float stage[kTok * kCh];                   // float32 latents of the next tile, as they are in global memory
     unsigned long long w1_full[kW1Stages], w1_free[kW1Stages], w2_full[kW2Stages], w2_free[kW2Stages];
-    unsigned long long stage_full, first_a, a_full[2], a_empty[2], d1_full[2], d1_empty[2], h_full[2], h_free[2], d2_full[2], d2_empty[2];
+    unsigned long long stage_full, first_a, a_full[2], a_empty[2], d1_full[kBufs], h_full[kBufs], buf_free[kBufs], d2_full[2], d2_empty[2];
     unsigned long long part_done, part_verdict;   // split mode: all epilogue warps have stored their partials / the ticket is drawn
     int is_last_part;
     uint32_t tmem_base;
@@ -105,9 +105,9 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
         if ((polls & 63u) == 0u) {
             if (*abort_flag) return false;
@@ -321,10 +321,11 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             mbar_init(&sm.a_empty[q], 1);
             mbar_init(&sm.d2_full[q], 1);
             mbar_init(&sm.d2_empty[q], kEpiWarps);
+        }
+        for (int q = 0; q < kBufs; ++q) {
             mbar_init(&sm.d1_full[q], 1);
-            mbar_init(&sm.d1_empty[q], kGroupWarps);
             mbar_init(&sm.h_full[q], kGroupWarps);
-            mbar_init(&sm.h_free[q], 1);
+            mbar_init(&sm.buf_free[q], 1);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -383,29 +384,30 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         const uint32_t a_lo = desc_lo(sm.a[0]), w1_lo = desc_lo(sm.w1[0]);
         bool ok = true;
         Ring<kW1Stages> r;        // weights of the next GEMM1
-        int g = 0;                // chunks issued so far: D1 buffer g & 1, its use number g >> 1
+        Ring<kBufs> cb;           // chunk buffer of the next GEMM1: slot = chunk mod 3, phase = parity of its use number
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int ab = it & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.a_full[ab], static_cast<uint32_t>(it >> 1) & 1u, abort_flag) ? 1 : 0) != 0;
             const uint32_t a_cur = a_lo + static_cast<uint32_t>(ab) * kTileUnits;
-            for (int c = 0; c < NC && ok; ++c, ++g) {       // D1[g & 1] = A * W1[r]
+            for (int c = 0; c < NC && ok; ++c) {            // D1[cb] = A * W1[r]
                 ok = mbar_wait(&sm.w1_full[r.slot], r.phase, abort_flag);
-                if (ok && g >= 2)      // the epilogue group of this parity has loaded chunk g - 2
-                    ok = mbar_wait(&sm.d1_empty[g & 1], static_cast<uint32_t>((g >> 1) - 1) & 1u, abort_flag);
+                if (ok && cb.wrapped)  // GEMM2 of the chunk that used this buffer three chunks ago has read its activations
+                    ok = mbar_wait(&sm.buf_free[cb.slot], cb.phase ^ 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t b_lo = w1_lo + static_cast<uint32_t>(r.slot) * kTileUnits;
-                const uint32_t d = tmem + static_cast<uint32_t>(g & 1) * kHc;
+                const uint32_t d = tmem + static_cast<uint32_t>(cb.slot) * kHc;
                 if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < kCh / 16; ++k)      // +32 bytes (2 descriptor units) per K step inside the swizzled row
                         umma_bf16(d, desc64(a_cur + 2u * k), desc64(b_lo + 2u * k), idesc1, k > 0 ? 1u : 0u);
-                    umma_commit(&sm.d1_full[g & 1]);
+                    umma_commit(&sm.d1_full[cb.slot]);
                     umma_commit(&sm.w1_free[r.slot]);
                 }
                 __syncwarp();
                 r.advance();
+                cb.advance();
             }
             if (ok && elect_one()) umma_commit(&sm.a_empty[ab]);       // every GEMM1 of this tile has been issued
             __syncwarp();
@@ -417,29 +419,31 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         const uint32_t w2_lo = desc_lo(sm.w2[0]);
         bool ok = true;
         Ring<kW2Stages> rw;       // weights of the next GEMM2
-        int g = 0;
+        Ring<kBufs> cb;           // chunk buffer of the next GEMM2
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            for (int c = 0; c < NC && ok; ++c, ++g) {       // D2 += H[g & 1] * W2[rw]
+            for (int c = 0; c < NC && ok; ++c) {            // D2 += H[cb] * W2[rw]
                 ok = mbar_wait(&sm.w2_full[rw.slot], rw.phase, abort_flag);
-                if (ok) ok = mbar_wait(&sm.h_full[g & 1], static_cast<uint32_t>(g >> 1) & 1u, abort_flag);
+                if (ok) ok = mbar_wait(&sm.h_full[cb.slot], cb.phase, abort_flag);
                 if (ok && c == 0 && it >= 2)      // the tile that used this D2 buffer two tiles ago has been written out
                     ok = mbar_wait(&sm.d2_empty[it & 1], static_cast<uint32_t>((it >> 1) - 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t h_col = tmem + kHCol + static_cast<uint32_t>(g & 1) * (kHc / 2);
+                const uint32_t h_col = tmem + static_cast<uint32_t>(cb.slot) * kHc;
                 const uint32_t wb_lo = w2_lo + static_cast<uint32_t>(rw.slot) * kTileUnits;
                 if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < kHc / 16; ++k)      // hidden 16k .. 16k+15 of the chunk: packed columns 8k .. 8k+7
-                        umma_bf16_ts(tmem + kD2Col + static_cast<uint32_t>(it & 1) * kCh, h_col + 8u * k,
+                    for (int k = 0; k < kHc / 16; ++k)      // hidden 16k .. 16k+15 of the chunk: 8 packed columns, the chunk's
+                                                            // first 64 hidden units at columns 0..31 of the buffer, the rest at 64..95
+                        umma_bf16_ts(tmem + kD2Col + static_cast<uint32_t>(it & 1) * kCh, h_col + (k / 4) * 64u + 8u * (k % 4),
                                      desc64(wb_lo + (k / 4) * ((kCh * 128) >> 4) + 2u * (k % 4)), idesc2, (c > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&sm.h_free[g & 1]);
+                    umma_commit(&sm.buf_free[cb.slot]);
                     umma_commit(&sm.w2_free[rw.slot]);
                     if (c == NC - 1) umma_commit(&sm.d2_full[it & 1]);
                 }
                 __syncwarp();
                 rw.advance();
+                cb.advance();
             }
         }
     } else if (warp == kLoaderWarp) {
@@ -612,41 +616,35 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
                     xb[m] = pack_bf16(gelu_x2(__uint_as_float(xb[m] << 16)), gelu_x2(__uint_as_float(xb[m] & 0xffff0000u)));
             }
         };
-        const uint32_t d1_slice = tmem + lane_addr + static_cast<uint32_t>(group) * kHc + (sub & 1u) * 64u;              // 64 fp32 columns
-        const uint32_t h_slice = tmem + lane_addr + kHCol + static_cast<uint32_t>(group) * (kHc / 2) + (sub & 1u) * 32u;  // 32 packed columns
+        const uint32_t my_cols = tmem + lane_addr + (sub & 1u) * 64u;     // this warp's 64 columns inside a chunk buffer
 
         uint32_t acc[32], xb[32];
-        int g = group;                // chunk index within this CTA's sequence of tiles x chunks; use number g >> 1 of the buffers
-        if (g < n_my_chunks)
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], 0u, abort_flag) ? 1 : 0) != 0;
-        for (; g < n_my_chunks && ok; g += 2) {
+        // chunk index within this CTA's sequence of tiles x chunks; its buffer is g mod 3, the buffer's use number g / 3
+        int buf = group, use = 0;
+        for (int g = group; g < n_my_chunks && ok; g += 2) {
             // tiles whose last GEMM2 was issued at least two chunks ago
             while (ok && (next_out + 1) * NC + 2 <= g) ok = output_tile(next_out++);
             if (!ok) break;
-            const uint32_t use = static_cast<uint32_t>(g >> 1);
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[buf], static_cast<uint32_t>(use) & 1u, abort_flag) ? 1 : 0) != 0;
+            if (!ok) break;
+            const uint32_t slice = my_cols + static_cast<uint32_t>(buf) * kHc;
             tc_fence_after();
-            tmem_ld32(d1_slice, acc);
+            tmem_ld32(slice, acc);
             tmem_ld_wait32(acc);
             pack16(acc, xb);
-            tmem_ld32(d1_slice + 32u, acc);
+            tmem_ld32(slice + 32u, acc);
             tmem_ld_wait32(acc);
             pack16(acc, xb + 16);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.d1_empty[group]);  // D1 of this chunk is in registers: GEMM1 of chunk g + 2 may go
             activate(xb);
-            if (g >= 2)       // the GEMM2 that read this group's previous activations must be done before they are overwritten
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.h_free[group], (use - 1u) & 1u, abort_flag) ? 1 : 0) != 0;
-            if (!ok) break;
-            tc_fence_after();
-            tmem_st16(h_slice, reinterpret_cast<const uint32_t (&)[16]>(xb[0]));
-            tmem_st16(h_slice + 16u, reinterpret_cast<const uint32_t (&)[16]>(xb[16]));
+            // the packed activations go over the first 32 of the 64 columns this warp has just read
+            tmem_st16(slice, reinterpret_cast<const uint32_t (&)[16]>(xb[0]));
+            tmem_st16(slice + 16u, reinterpret_cast<const uint32_t (&)[16]>(xb[16]));
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.h_full[group]);
-            if (g + 2 < n_my_chunks)
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.d1_full[group], (use + 1u) & 1u, abort_flag) ? 1 : 0) != 0;
+            if (lane == 0) mbar_arrive(&sm.h_full[buf]);
+            buf += 2;
+            if (buf >= kBufs) { buf -= kBufs; ++use; }
         }
         while (ok && next_out < n_my_tiles) ok = output_tile(next_out++);
         tmem_ld_wait();
