@@ -241,25 +241,28 @@ __device__ __forceinline__ uint32_t bf2_fma(uint32_t a, uint32_t b, uint32_t c) 
     asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
-// Twice the erf-form GELU for |x| < 2 without a special-function instruction:
+// Twice the erf-form GELU for |x| < 1.5 without a special-function instruction:
 //     2 GELU(x) = x + x erf(x / sqrt 2) = x + s Q(s),   s = x^2,
-// with Q a cubic in s fitted to erf(x / sqrt 2) / x on [0, 2] (minimax in s Q(s), the coefficients rounded to bf16 one
-// after the other and the rest refitted; the error of the polynomial itself is 2.1e-4 absolute).  Evaluated on a packed
-// pair in bf16: one multiply and four fused multiply-adds on the FMA pipe, where the hardware tanh allows sixteen
-// activations per clock and SM and so bounds the whole stage at twice the tensor-core time.  The last operation,
-// fma(t, s, x), adds the small even part to x and rounds once, so for the usual |x| << 1 the result differs from the
-// correctly rounded activation by the rounding of x to bf16 and little else.
-constexpr uint32_t kGeluQ0 = 0x3f4c3f4cu;   //  0.796875
-constexpr uint32_t kGeluQ1 = 0xbe04be04u;   // -0.12890625
-constexpr uint32_t kGeluQ2 = 0x3c843c84u;   //  0.01611328125
-constexpr uint32_t kGeluQ3 = 0xba7dba7du;   // -0.000965118408203125
-constexpr uint32_t kGeluRangeBits = 0x40004000u;   // exponent bit of bf16 that is set exactly when |x| >= 2 (or x is not finite)
+// with Q a quadratic in s fitted to erf(x / sqrt 2) / x on [0, 1.5] (minimax in s Q(s), the coefficients rounded to bf16
+// one after the other and the rest refitted by csrc/gelu_poly_fit.py; the polynomial is within 6.3e-4 of the function).
+// Evaluated on a packed pair in bf16: one multiply and three fused multiply-adds on the FMA pipe, where one hardware
+// tanh per activation (sixteen per clock and SM) bounds the whole stage at twice the tensor-core time.  The last
+// operation, fma(t, s, x), adds the small even part to x and rounds once, so for the usual |x| << 1 the result differs
+// from the correctly rounded activation by the rounding of x to bf16 and little else.
+constexpr uint32_t kGeluQ0 = 0x3f4b3f4bu;   //  0.79296875
+constexpr uint32_t kGeluQ1 = 0xbdf8bdf8u;   // -0.12109375
+constexpr uint32_t kGeluQ2 = 0x3c383c38u;   //  0.01123046875
+constexpr uint32_t kGeluRangeBf16 = 0x3fc0u;   // bf16 bits of 1.5: the polynomial's range
 __device__ __forceinline__ uint32_t gelu_x2_poly(uint32_t xb) {
     const uint32_t s = bf2_mul(xb, xb);
-    uint32_t t = bf2_fma(kGeluQ3, s, kGeluQ2);
-    t = bf2_fma(t, s, kGeluQ1);
+    uint32_t t = bf2_fma(kGeluQ2, s, kGeluQ1);
     t = bf2_fma(t, s, kGeluQ0);
     return bf2_fma(t, s, xb);
+}
+// Running maximum of magnitudes over packed pairs (the sign bits of the result carry no meaning).
+__device__ __forceinline__ uint32_t bf2_absmax(uint32_t m, uint32_t x) {
+    asm("max.xorsign.abs.bf16x2 %0, %0, %1;" : "+r"(m) : "r"(x));
+    return m;
 }
 // byte offset of the 16-byte piece `c16` of row r inside a 128-byte-swizzled tile of 128-byte rows
 __device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c16) { return r * 128u + ((c16 ^ (r & 7u)) << 4); }
@@ -351,11 +354,13 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
 
     if (warp == 0) {
         // ---------------------------------------------------------------- weight producers (lane 0: W1, lane 1: W2)
-        // The sum over hidden chunks may be taken in any order; each CTA starts at its own chunk so that the SMs do
-        // not all ask the same L2 lines for the same chunk at the same moment.
+        // Every tile adds its hidden chunks in index order, whatever CTA it lands on, so a token's output does not
+        // depend on how many tokens the launch holds (a shard of a batch reproduces the batch's bits as long as neither
+        // launch is cut along the hidden dimension).  Starting every CTA at its own chunk instead, to spread the L2
+        // requests, measured the same.
         if (lane == 0) {
             Ring<kW1Stages> r;
-            int cc = cta % NC;
+            int cc = 0;
             for (int g = 0; g < n_my_chunks; ++g) {
                 if (r.wrapped && !mbar_wait(&sm.w1_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM1 that read this slot is done
                 mbar_expect_tx(&sm.w1_full[r.slot], kTileBytes);
@@ -365,7 +370,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             }
         } else if (lane == 1) {
             Ring<kW2Stages> r;
-            int cc = cta % NC;
+            int cc = 0;
             for (int g = 0; g < n_my_chunks; ++g) {
                 if (r.wrapped && !mbar_wait(&sm.w2_free[r.slot], r.phase ^ 1u, abort_flag)) break;    // GEMM2 that read this slot is done
                 mbar_expect_tx(&sm.w2_full[r.slot], kTileBytes);
@@ -595,8 +600,8 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         // 32 accumulator columns -> 16 registers of packed bf16 activation pairs
         // One chunk of this warp: 64 accumulator columns arrive as float32, are rounded to packed bf16 pairs at once (32
         // registers) and D1 is handed back before any arithmetic, so GEMM1 of chunk g + 2 runs under the activation of
-        // chunk g.  The packed polynomial covers |x| < 2; the OR of the packed inputs shows whether any of this thread's
-        // 64 values lies outside (its top exponent bit is set), and only then the thread takes the hardware-tanh form
+        // chunk g.  The packed polynomial covers |x| < 1.5; a running maximum of magnitudes shows whether any of this
+        // thread's 64 values lies outside (or is not finite), and only then the thread takes the hardware-tanh form
         // for its values.  With weights and latents of the usual scale (pre-activations of standard deviation ~0.2) that
         // never happens.
         auto pack16 = [&](const uint32_t (&acc)[32], uint32_t* xb) {
@@ -604,10 +609,10 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
             for (int m = 0; m < 16; ++m) xb[m] = pack_bf16(__uint_as_float(acc[2 * m]), __uint_as_float(acc[2 * m + 1]));
         };
         auto activate = [&](uint32_t (&xb)[32]) {
-            uint32_t seen = 0u;
+            uint32_t big = 0u;
 #pragma unroll
-            for (int m = 0; m < 32; ++m) seen |= xb[m];
-            if (!(seen & kGeluRangeBits)) {
+            for (int m = 0; m < 32; ++m) big = bf2_absmax(big, xb[m]);
+            if ((big & 0x7fffu) < kGeluRangeBf16 && ((big >> 16) & 0x7fffu) < kGeluRangeBf16) {
 #pragma unroll
                 for (int m = 0; m < 32; ++m) xb[m] = gelu_x2_poly(xb[m]);
             } else {
