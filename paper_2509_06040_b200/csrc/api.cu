@@ -174,6 +174,7 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     t->D = static_cast<int64_t>(desc->tokens) * desc->channels;
     t->nchunks = nchunks_of(t->D);
     t->nchunks_step = nchunks_step_of(t->D);
+    t->nchunks_reward = static_cast<int32_t>((t->D / 4 + kRewardChunkVec - 1) / kRewardChunkVec);
     t->independent = !(std::isfinite(desc->branch_corr_s) && desc->branch_corr_s >= 0.0f);
     if (t->independent) {
         t->mix_shared = 0.0f;
@@ -411,7 +412,7 @@ static bgrpo_status reward_common(bgrpo_tree* t, const float* target, float scal
     p.D = t->D;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
-    p.nchunks = t->nchunks;
+    p.nchunks = t->nchunks_reward;
     p.leaves = t->lv.width[t->desc.T];
     p.off_leaf = t->lv.offset[t->desc.T];
     p.scale = scale;
@@ -500,7 +501,6 @@ bgrpo_status bgrpo_tree_prune(bgrpo_tree* t, int32_t width_mode, int32_t k_or_b,
     for (int i = 0; i < t->desc.T; ++i)
         if (t->lv.fanout[i] > 1) p.last_split = i;
     p.ignore_last = ignore_last_step ? 1 : 0;
-    if (static_cast<size_t>(p.nodes) > 200 * 1024) return fail(BGRPO_ERR_UNSUPPORTED, "tree too large for one CTA's shared memory");
     cudaError_t e = launch_prune(p, as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "prune kernel");
     return BGRPO_OK;

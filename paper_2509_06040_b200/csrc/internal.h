@@ -10,7 +10,9 @@
 namespace bgrpo {
 
 constexpr int kStreamThreads = 256;    // threads per CTA of the root / reward kernels
-constexpr int kChunkVec = 1024;        // float4 per (row, chunk) work item of the root / reward kernels
+constexpr int kChunkVec = 1024;        // float4 per (row, chunk) work item of the root kernel
+constexpr int kRewardVec = 16;         // float4 of a row per thread of the leaf-reward kernel
+constexpr int kRewardChunkVec = kStreamThreads * kRewardVec;   // float4 per (row, chunk) work item of the leaf-reward kernel
 // Step kernel: 64-thread CTAs, 8 float4 per thread.  Measured on B200 against 128/256-thread CTAs, 2/4/6 float4 per
 // thread, persistent grids and a shared-memory ring fed by bulk asynchronous copies: the kernel is bound by
 // instruction issue (Philox + Box-Muller), and eight independent noise chains per thread with many small CTAs
@@ -97,7 +99,8 @@ struct bgrpo_tree {
     uint64_t ode_bits;                   // bit i set: step i is an ODE step of the hybrid schedule (sigma = 0)
     int32_t depth;                       // steps taken so far
     int64_t D;                           // elements per node
-    int32_t nchunks;                     // reward / root work items per node row
+    int32_t nchunks;                     // root-kernel work items per node row (also sizes the reward partials)
+    int32_t nchunks_reward;              // leaf-reward work items per node row
     int32_t nchunks_step;                // step-kernel work items per node row
     bool independent;                    // s = inf: xi_b = eta_b
     float mix_shared, mix_innov;         // xi_b = mix_shared*xi_0 + mix_innov*eta_b

@@ -1,5 +1,5 @@
 // Tree reductions: reward fusion (Eq. 3) + depth-wise normalisation (Eq. 4) in one kernel, and the width / depth
-// pruning masks ("Pruning Strategies") in another.  A tree has at most a few thousand nodes, so one CTA owns one
+// pruning masks ("Pruning Strategies") in another.  A tree usually has at most a few thousand nodes, so one CTA owns one
 // tree, keeps the per-node state in shared memory as doubles and walks the levels; the kernels are latency-bound.
 // A tree whose per-node state does not fit in shared memory (more than about 8 500 nodes: K = 4 with seven splits, say)
 // keeps it in the caller's scratch instead; the code is the same, only the pointer differs.
@@ -156,40 +156,87 @@ fusion_ess_kernel(const EssLaunch p) {
     }
 }
 
-// rank of x among its siblings / leaves: number of entries that beat it (larger value, or equal value and lower index)
+// rank of x among its siblings: number of entries that beat it (larger value, or equal value and lower index)
 __device__ __forceinline__ bool beats(float v_other, int i_other, float v_me, int i_me) {
     return (v_other > v_me) || (v_other == v_me && i_other < i_me);
+}
+
+// Sort keys of the Extreme-b selection.  A float32 maps to an unsigned integer of the same order (sign bit flipped for
+// non-negative values, all bits for negative ones); the leaf index goes below it, complemented, so that among equal
+// values the lower index has the larger key.  "best" ranks large values first, "worst" small values first: the b
+// leaves with the largest keys are the ones the ranking "value, ties to the lower leaf index" puts first.
+__device__ __forceinline__ uint64_t extreme_key(float v, uint32_t leaf, bool worst) {
+    uint32_t u = __float_as_uint(v);
+    if ((u << 1) == 0u) u = 0u;                              // -0 and +0 compare equal
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    if (worst) u = ~u;
+    return (static_cast<uint64_t>(u) << 32) | static_cast<uint64_t>(~leaf);
+}
+
+// The want-th largest key among the tree's leaves (1 <= want <= L): radix selection, eight passes of eight bits over
+// the 64-bit keys; every pass histograms the keys that share the prefix fixed so far.  Keys are distinct (they hold
+// the leaf index), so exactly `want` leaves have a key >= the result.  Called by the whole CTA.
+__device__ uint64_t select_kth_largest(const float* leaf_vals, int L, int want, bool worst, unsigned int* hist, uint64_t* shared_prefix,
+                                       int* shared_want) {
+    if (threadIdx.x == 0) { *shared_prefix = 0; *shared_want = want; }
+    for (int pass = 7; pass >= 0; --pass) {
+        for (int i = threadIdx.x; i < 256; i += kTreeThreads) hist[i] = 0u;
+        __syncthreads();
+        const uint64_t prefix = *shared_prefix;
+        const int shift = 8 * pass;
+        for (int l = threadIdx.x; l < L; l += kTreeThreads) {
+            const uint64_t key = extreme_key(leaf_vals[l], static_cast<uint32_t>(l), worst);
+            const bool same_prefix = (pass == 7) || ((key >> (shift + 8)) == (prefix >> (shift + 8)));
+            if (same_prefix) atomicAdd(&hist[static_cast<unsigned int>(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int left = *shared_want, bin = 255;
+            for (; bin > 0; --bin) {                        // bins from the largest digit down
+                const int c = static_cast<int>(hist[bin]);
+                if (c >= left) break;
+                left -= c;
+            }
+            *shared_want = left;
+            *shared_prefix = prefix | (static_cast<uint64_t>(bin) << shift);
+        }
+        __syncthreads();
+    }
+    return *shared_prefix;
 }
 
 __global__ void __launch_bounds__(kTreeThreads)
 prune_kernel(const PruneLaunch p) {
     pdl_release();
     pdl_wait();
-    extern __shared__ unsigned char keep[];            // per node, then (small trees) the node values as floats
+    extern __shared__ unsigned char prune_smem[];      // small trees: the node values as floats
     const int tree = blockIdx.x;
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     const int T = p.T;
     const float* rbar = p.rbar + row0;
     if (p.values_in_smem) {        // fetched once: a level then waits for no global load
-        float* vals = reinterpret_cast<float*>(keep + ((static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15)));
+        float* vals = reinterpret_cast<float*>(prune_smem);
         for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) vals[n] = rbar[n];
         rbar = vals;
         __syncthreads();
     }
     if (p.mode == BGRPO_WIDTH_EXTREME_B) {
+        // The mask itself holds the keep flags while they are gathered: 0 everywhere, 1 on the root paths of the
+        // selected leaves (several threads may write the same 1), then the depth conditions are applied in place.
+        __shared__ unsigned int hist[256];
+        __shared__ uint64_t s_prefix;
+        __shared__ int s_want;
+        uint8_t* keep = p.mask + row0;
         for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) keep[n] = 0;
-        __syncthreads();
         const int L = p.lv.width[T], off = p.lv.offset[T];
-        const int64_t rows = static_cast<int64_t>(p.n_trees) * p.nodes_cap;
+        const int want = p.k < L ? p.k : L;
+        const uint64_t best_cut = select_kth_largest(rbar + off, L, want, false, hist, &s_prefix, &s_want);
+        __syncthreads();
+        const uint64_t worst_cut = select_kth_largest(rbar + off, L, want, true, hist, &s_prefix, &s_want);
+        __syncthreads();                                   // also orders the zero fill before the flags below
         for (int l = threadIdx.x; l < L; l += kTreeThreads) {
             const float v = rbar[off + l];
-            int better = 0, worse = 0;
-            for (int q = 0; q < L; ++q) {
-                const float u = rbar[off + q];
-                better += beats(u, q, v, l) ? 1 : 0;                       // rank from the top
-                worse += ((u < v) || (u == v && q < l)) ? 1 : 0;           // rank from the bottom
-            }
-            if (better < p.k || worse < p.k) {
+            if (extreme_key(v, static_cast<uint32_t>(l), false) >= best_cut || extreme_key(v, static_cast<uint32_t>(l), true) >= worst_cut) {
                 int n = off + l;
                 for (int guard = 0; n >= 0 && guard <= T; ++guard) {       // root path through the node table
                     keep[n] = 1;
@@ -197,45 +244,43 @@ prune_kernel(const PruneLaunch p) {
                 }
             }
         }
-        (void)rows;
         __syncthreads();
-    } else {
-        // Top-k modes: a node is kept iff, at every ranked split on its root path, the ancestor (or the node itself)
-        // ranks among the k best of its siblings.  Every node walks its own path (children of the j-th node of depth d
-        // are j*F + b of depth d+1, so the parent of j is j / F): no level-by-level pass, no barrier.
-        __shared__ int s_off[BGRPO_MAX_T + 2], s_fan[BGRPO_MAX_T];
-        for (int i = threadIdx.x; i <= T + 1; i += kTreeThreads) s_off[i] = p.lv.offset[i];
-        for (int i = threadIdx.x; i < T; i += kTreeThreads) s_fan[i] = p.lv.fanout[i];
-        __syncthreads();
-        for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) {       // one node per thread, all depths at once
-            int d = 0;
-            while (d < T && n >= s_off[d + 1]) ++d;
+        for (int d = 0; d <= T; ++d) {
             const bool depth_ok = d > 0 && !((p.pruned_bits >> (d - 1)) & 1ull) && !(p.ignore_last && d == T);
-            bool kept = true;
-            int j = n - s_off[d];
-            for (int e = d; e > 0 && kept; --e) {                // e: depth of the node j on the path
-                const int fan = s_fan[e - 1];
-                const int pj = j / fan, b = j - pj * fan;
-                const bool ranked = fan > 1 && (p.mode == BGRPO_WIDTH_PER_SPLIT_TOPK ||
-                                                (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && e - 1 == p.last_split));
-                if (ranked) {
-                    const int sib0 = s_off[e] + pj * fan;
-                    const float v = rbar[sib0 + b];
-                    int rank = 0;
-                    for (int q = 0; q < fan; ++q) rank += beats(rbar[sib0 + q], q, v, b) ? 1 : 0;
-                    kept = rank < p.k;
-                }
-                j = pj;
-            }
-            p.mask[row0 + n] = (depth_ok && kept) ? 1 : 0;
+            const int offd = p.lv.offset[d];
+            for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads)
+                if (!depth_ok) keep[offd + j] = 0;
         }
         return;
     }
-    for (int d = 0; d <= T; ++d) {
+    // Top-k modes: a node is kept iff, at every ranked split on its root path, the ancestor (or the node itself)
+    // ranks among the k best of its siblings.  Every node walks its own path (children of the j-th node of depth d
+    // are j*F + b of depth d+1, so the parent of j is j / F): no level-by-level pass, no barrier.
+    __shared__ int s_off[BGRPO_MAX_T + 2], s_fan[BGRPO_MAX_T];
+    for (int i = threadIdx.x; i <= T + 1; i += kTreeThreads) s_off[i] = p.lv.offset[i];
+    for (int i = threadIdx.x; i < T; i += kTreeThreads) s_fan[i] = p.lv.fanout[i];
+    __syncthreads();
+    for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) {       // one node per thread, all depths at once
+        int d = 0;
+        while (d < T && n >= s_off[d + 1]) ++d;
         const bool depth_ok = d > 0 && !((p.pruned_bits >> (d - 1)) & 1ull) && !(p.ignore_last && d == T);
-        const int off = p.lv.offset[d];
-        for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads)
-            p.mask[row0 + off + j] = (depth_ok && keep[off + j]) ? 1 : 0;
+        bool kept = true;
+        int j = n - s_off[d];
+        for (int e = d; e > 0 && kept; --e) {                // e: depth of the node j on the path
+            const int fan = s_fan[e - 1];
+            const int pj = j / fan, b = j - pj * fan;
+            const bool ranked = fan > 1 && (p.mode == BGRPO_WIDTH_PER_SPLIT_TOPK ||
+                                            (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && e - 1 == p.last_split));
+            if (ranked) {
+                const int sib0 = s_off[e] + pj * fan;
+                const float v = rbar[sib0 + b];
+                int rank = 0;
+                for (int q = 0; q < fan; ++q) rank += beats(rbar[sib0 + q], q, v, b) ? 1 : 0;
+                kept = rank < p.k;
+            }
+            j = pj;
+        }
+        p.mask[row0 + n] = (depth_ok && kept) ? 1 : 0;
     }
 }
 
@@ -304,9 +349,9 @@ cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s) {
 
 cudaError_t launch_prune(const PruneLaunch& p0, cudaStream_t s) {
     PruneLaunch p = p0;
-    size_t smem = (static_cast<size_t>(p.nodes) + 15) & ~static_cast<size_t>(15);
-    p.values_in_smem = smem + static_cast<size_t>(p.nodes) * sizeof(float) <= kTreeSmemLimit ? 1 : 0;
-    if (p.values_in_smem) smem += static_cast<size_t>(p.nodes) * sizeof(float);
+    size_t smem = static_cast<size_t>(p.nodes) * sizeof(float);
+    p.values_in_smem = smem <= kTreeSmemLimit ? 1 : 0;       // larger trees read the values from global memory
+    if (!p.values_in_smem) smem = 0;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;

@@ -1,15 +1,15 @@
 // Leaf-reward stand-ins (Algorithm 1, "Evaluate rewards"; the paper's reward models are out of scope): streaming
-// reductions over the leaf rows.  Sums over a row are float32 inside a thread, double from the warp level on, one double
-// per (row, chunk, component), and the chunks are added in a fixed order by a small finish kernel.
+// reductions over the leaf rows.  Sums over a row are float32 over runs of sixteen elements, double from there on, one
+// double per (row, chunk, component), and the chunks are added in a fixed order by a small finish kernel.
 #include "internal.h"
 
 namespace bgrpo {
 namespace {
 
-constexpr int kVecPerThread = kChunkVec / kStreamThreads;   // 4
 constexpr int kWarps = kStreamThreads / 32;
 constexpr int kPartialStride = 3;                           // doubles per (row, chunk) slot
-constexpr int kPairs = 1;                                   // chunks per CTA of the reward kernel (1 and 2 measured the same)
+constexpr int kBatch = 8;                                   // float4 of each operand a thread has in flight at once
+constexpr int kBatches = kRewardVec / kBatch;
 
 __device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
@@ -29,79 +29,113 @@ __device__ __forceinline__ double row_total(const double* partials, int64_t row,
 
 // ---------------------------------------------------------------------------------------------------------------
 // Leaf rewards: mode 0  r = -mean (z - target)^2 ; mode 1  r += scale * cos(z, target).
+// One CTA per (leaf row, chunk of kRewardChunkVec float4 = 64 KiB of the row).  A thread takes sixteen float4 of the row
+// and of the target in two batches of eight; the sixteen 128-bit loads of a batch are issued before the first value is
+// used.  Sums are float32 over a run of sixteen elements (four float4), double from there on; the warp and CTA
+// reductions, in double, happen once per 64 KiB, so they cost a few per cent of the instructions instead of most of them.
+// 128-bit loads as volatile instructions: the compiler keeps the loads of a batch in program order, ahead of the
+// arithmetic that uses them, instead of sinking each load to its first use.  The leaf row is read once (evict first);
+// the target row is shared by all leaves of a tree (read-only path).
+__device__ __forceinline__ float4 load_streaming(const float4* p) {
+    float4 v;
+    asm volatile("ld.global.cs.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 load_shared_row(const float4* p) {
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// FULL: the chunk lies inside the row, no element needs a bounds test (so the loads of a batch are plain back-to-back
+// instructions the compiler keeps together).
+template <int MODE, bool FULL>
+__device__ __forceinline__ void accumulate_chunk(const float4* __restrict__ z, const float4* __restrict__ tg, uint32_t e0, uint32_t D4,
+                                                 double (&dsum)[(MODE == 0) ? 1 : 3]) {
+    constexpr int NV = (MODE == 0) ? 1 : 3;
+#pragma unroll
+    for (int h = 0; h < kBatches; ++h) {
+        float4 a[kBatch], t[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            const uint32_t e = e0 + static_cast<uint32_t>(h * kBatch + k) * kStreamThreads;
+            if (FULL || e < D4) {
+                a[k] = load_streaming(z + e);
+                t[k] = load_shared_row(tg + e);
+            } else {
+                a[k] = make_float4(0.f, 0.f, 0.f, 0.f);      // past the row: contributes nothing to any of the sums
+                t[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        if (FULL) {      // nothing below may move above the last load of the batch
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                asm volatile("" : "+f"(a[k].x), "+f"(a[k].y), "+f"(a[k].z), "+f"(a[k].w));
+                asm volatile("" : "+f"(t[k].x), "+f"(t[k].y), "+f"(t[k].z), "+f"(t[k].w));
+            }
+        }
+#pragma unroll
+        for (int run = 0; run < kBatch / 4; ++run) {         // sixteen elements in float32, then into the double
+            float acc[NV];
+#pragma unroll
+            for (int v = 0; v < NV; ++v) acc[v] = 0.0f;
+#pragma unroll
+            for (int k = run * 4; k < run * 4 + 4; ++k) {
+                const float av[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
+                const float tv[4] = {t[k].x, t[k].y, t[k].z, t[k].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (MODE == 0) {
+                        const float d = av[q] - tv[q];
+                        acc[0] = fmaf(d, d, acc[0]);
+                    } else {
+                        acc[0] = fmaf(av[q], tv[q], acc[0]);
+                        acc[1] = fmaf(av[q], av[q], acc[1]);
+                        acc[2] = fmaf(tv[q], tv[q], acc[2]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int v = 0; v < NV; ++v) dsum[v] += static_cast<double>(acc[v]);
+        }
+    }
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(kStreamThreads)
 reward_kernel(const __grid_constant__ RewardLaunch p) {
     pdl_release();
     pdl_wait();
-    // A CTA takes kPairs consecutive chunks of a row and issues all their loads before it touches a value.
-    const int npairs = (p.nchunks + kPairs - 1) / kPairs;
-    const int pair = blockIdx.x % npairs;
-    const int row = blockIdx.x / npairs;                // tree * leaves + l
+    const int chunk = blockIdx.x % p.nchunks;
+    const int row = blockIdx.x / p.nchunks;             // tree * leaves + l
     const int tree = row / p.leaves;
     const int l = row - tree * p.leaves;
-    const int64_t D4 = p.D >> 2;
+    const uint32_t D4 = static_cast<uint32_t>(p.D >> 2);
     const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + l;
     const float4* __restrict__ z = reinterpret_cast<const float4*>(p.latents + node_row * p.D);
     const float4* __restrict__ tg = reinterpret_cast<const float4*>(p.target + static_cast<int64_t>(tree) * p.D);
     constexpr int NV = (MODE == 0) ? 1 : 3;
-    float acc[kPairs][NV];
-    float4 a[kPairs][kVecPerThread], t[kPairs][kVecPerThread];
+    const uint32_t c0 = static_cast<uint32_t>(chunk) * kRewardChunkVec;
+    double dsum[NV];
 #pragma unroll
-    for (int h = 0; h < kPairs; ++h) {
-#pragma unroll
-        for (int v = 0; v < NV; ++v) acc[h][v] = 0.0f;
-        const int64_t e0 = static_cast<int64_t>(pair * kPairs + h) * kChunkVec + threadIdx.x;
-#pragma unroll
-        for (int k = 0; k < kVecPerThread; ++k) {
-            const int64_t e = e0 + k * kStreamThreads;
-            if (e < D4) { a[h][k] = __ldcs(z + e); t[h][k] = __ldg(tg + e); }
-        }
-    }
-#pragma unroll
-    for (int h = 0; h < kPairs; ++h) {
-        const int64_t e0 = static_cast<int64_t>(pair * kPairs + h) * kChunkVec + threadIdx.x;
-#pragma unroll
-        for (int k = 0; k < kVecPerThread; ++k) {
-            const int64_t e = e0 + k * kStreamThreads;
-            if (e < D4) {
-                const float av[4] = {a[h][k].x, a[h][k].y, a[h][k].z, a[h][k].w};
-                const float tv[4] = {t[h][k].x, t[h][k].y, t[h][k].z, t[h][k].w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (MODE == 0) {
-                        const float d = av[q] - tv[q];
-                        acc[h][0] = fmaf(d, d, acc[h][0]);
-                    } else {
-                        acc[h][0] = fmaf(av[q], tv[q], acc[h][0]);
-                        acc[h][1] = fmaf(av[q], av[q], acc[h][1]);
-                        acc[h][2] = fmaf(tv[q], tv[q], acc[h][2]);
-                    }
-                }
-            }
-        }
-    }
-    // One double per (row, chunk, component): thread sums are float over 16 elements, double from the warp level on.
-    // Nothing waits for these stores; reward_finish_kernel, next on the stream, adds the chunks up in order.
-    __shared__ double red[kPairs * NV][kWarps];
+    for (int v = 0; v < NV; ++v) dsum[v] = 0.0;
+    if (c0 + kRewardChunkVec <= D4) accumulate_chunk<MODE, true>(z, tg, c0 + threadIdx.x, D4, dsum);
+    else accumulate_chunk<MODE, false>(z, tg, c0 + threadIdx.x, D4, dsum);
+    // One double per (row, chunk, component).  Nothing waits for these stores; reward_finish_kernel, next on the
+    // stream, adds the chunks up in order.
+    __shared__ double red[NV][kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-    for (int h = 0; h < kPairs; ++h)
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const double s = warp_sum(static_cast<double>(acc[h][v]));
-            if (lane == 0) red[h * NV + v][warp] = s;
-        }
+    for (int v = 0; v < NV; ++v) {
+        const double s = warp_sum(dsum[v]);
+        if (lane == 0) red[v][warp] = s;
+    }
     __syncthreads();
-    if (threadIdx.x < kPairs * NV) {
-        const int h = threadIdx.x / NV, v = threadIdx.x - h * NV;
-        const int chunk = pair * kPairs + h;
-        if (chunk < p.nchunks) {
-            double s = 0.0;
+    if (threadIdx.x < NV) {
+        double s = 0.0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
-            p.partials[(node_row * p.nchunks + chunk) * kPartialStride + v] = s;
-        }
+        for (int w = 0; w < kWarps; ++w) s += red[threadIdx.x][w];
+        p.partials[(node_row * p.nchunks + chunk) * kPartialStride + threadIdx.x] = s;
     }
 }
 
@@ -130,7 +164,7 @@ reward_finish_kernel(const __grid_constant__ RewardLaunch p) {
 }  // namespace
 
 cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s) {
-    const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * ((p.nchunks + kPairs - 1) / kPairs);
+    const int64_t items = static_cast<int64_t>(p.n_trees) * p.leaves * p.nchunks;
     if (items <= 0 || items > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const unsigned int rows = static_cast<unsigned int>(p.n_trees) * static_cast<unsigned int>(p.leaves);
     const unsigned int fgrid = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);

@@ -633,3 +633,38 @@ def test_reductions_on_a_tree_larger_than_shared_memory(B):
     assert np.all(np.abs(ess.cpu().numpy()[t] - ref_ess) <= 1e-5 * ref_ess)
     mask = credit.gradient_mask(topo, s.rbar.cpu().numpy()[t], B.WIDTH_PER_SPLIT_TOPK, 2, (1, 4), False)
     assert np.array_equal(s.mask.cpu().numpy()[t], mask)
+    # Extreme-b on the 16 384 leaves of this tree (a CTA-wide selection of the b-th best and b-th worst leaf), with
+    # exact ties: values rounded to one decimal, signed zeros included
+    coarse = np.round(s.rbar.cpu().numpy(), 1).astype(np.float32)
+    s.rbar.copy_(torch.from_numpy(coarse))
+    for b, pruned, ign in ((1, (), False), (37, (2,), True), (5000, (), False), (10 ** 6, (0, 6), False)):
+        s.mask.fill_(9)
+        B.tree_prune(s.tree, B.WIDTH_EXTREME_B, b, pruned, ign)
+        torch.cuda.synchronize()
+        got = s.mask.cpu().numpy()
+        for t in range(2):
+            ref = credit.gradient_mask(topo, coarse[t], B.WIDTH_EXTREME_B, b, pruned, ign)
+            assert np.array_equal(got[t], ref), (b, t)
+            if not pruned and not ign:
+                assert int(got[t][list(topo.leaf_ids())].sum()) == min(2 * b, topo.leaves)
+
+
+def test_prune_has_no_node_limit(B):
+    """A tree of 349 525 nodes (K = 4, nine splits): every pruning mode runs (the values stay in global memory, the
+    Extreme-b flags are gathered in the mask itself) and matches the oracle."""
+    T, K, splits = 9, 4, tuple(range(9))
+    w = Workload(name="huge9", n_trees=1, tokens=1, channels=4, T=T, K=K, splits=splits, sigma=0.3,
+                 velocity="linear", reward="neg_mse_mu")
+    s = _session(w)
+    s.upload_inputs(make_inputs(w))
+    s.rollout()
+    topo = otree.build_topology(T, K, splits)
+    assert topo.nodes == 349525
+    rng = np.random.default_rng(5)
+    rbar = np.round(rng.standard_normal((1, topo.nodes)), 2).astype(np.float32)
+    s.rbar.copy_(torch.from_numpy(rbar))
+    for mode, k in ((B.WIDTH_EXTREME_B, 3), (B.WIDTH_LAST_SPLIT_TOPK, 1)):
+        B.tree_prune(s.tree, mode, k, (4,), False)
+        torch.cuda.synchronize()
+        ref = credit.gradient_mask(topo, rbar[0], mode, k, (4,), False)
+        assert np.array_equal(s.mask.cpu().numpy()[0], ref), mode
