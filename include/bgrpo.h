@@ -234,9 +234,18 @@ bgrpo_status bgrpo_tree_stats(const bgrpo_tree* tree, int32_t* depth, int64_t* n
 /* Level layout: writes min(depth+1, n) widths and offsets (host arrays). */
 bgrpo_status bgrpo_tree_levels(const bgrpo_tree* tree, int32_t n, int32_t* widths_out, int32_t* offsets_out);
 
-/* Copies the device status word to the host and waits for `stream`: BGRPO_OK, BGRPO_ERR_NONFINITE, or
- * BGRPO_ERR_CUDA.  The word is cleared afterwards. */
+/* Copies the device status word to the host and waits for `stream`: BGRPO_OK, BGRPO_ERR_NONFINITE (a kernel met a
+ * NaN/Inf leaf reward), BGRPO_ERR_CUDA (a bounded wait inside the MLP velocity kernel ran out) or, in the debug build,
+ * BGRPO_ERR_CAPACITY (a device-side index check failed; the access was skipped).  The word is cleared afterwards. */
 bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* tree, void* stream);
+
+/* Debug build with device-side index checks (library compiled with -DBGRPO_DEBUG_BOUNDS; no counterpart in the paper).
+ * In that build every kernel tests the row, chunk and element indices it derives against the extents it was launched
+ * with; a failed test sets a bit of the status word and the access is skipped - nothing traps - and
+ * bgrpo_tree_sync_status then returns BGRPO_ERR_CAPACITY.  bgrpo_debug_bounds returns BGRPO_OK in such a build and
+ * BGRPO_ERR_UNSUPPORTED in the normal one; with trip != 0 it also enqueues a one-warp kernel that fails one such test on
+ * purpose (it touches no memory), so the reporting path can be checked. */
+bgrpo_status bgrpo_debug_bounds(bgrpo_tree* tree, int32_t trip, void* stream);
 
 /* Test hooks for the noise definition above: raw Philox words (n_blocks x 4 uint32) and normals (n floats,
  * n % 4 == 0) of one (seed, node id, step, tag), starting at element 0. */

@@ -18,7 +18,9 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbgrpo.so")
+# BGRPO_DEBUG_BOUNDS=1 selects the build whose kernels check every index they derive (python -m ...build --debug-bounds)
+DEBUG_BOUNDS = os.environ.get("BGRPO_DEBUG_BOUNDS", "0") == "1"
+LIB_PATH = os.path.join(_HERE, "libbgrpo_debug.so" if DEBUG_BOUNDS else "libbgrpo.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -83,6 +85,7 @@ _SIGNATURES = {
     "bgrpo_philox_words_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
     "bgrpo_philox_normal_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
     "bgrpo_reward_mse_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p]),
+    "bgrpo_debug_bounds": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "bgrpo_tree_destroy": (None, [C.c_void_p]),
     "bgrpo_status_string": (C.c_char_p, [C.c_int]),
     "bgrpo_last_error": (C.c_char_p, []),
@@ -261,6 +264,11 @@ def tree_levels(tree: Tree):
 
 def tree_sync_status(tree: Tree, stream=None):
     _check(lib.bgrpo_tree_sync_status(tree.handle, _stream(stream)), "bgrpo_tree_sync_status")
+
+
+def debug_bounds(tree: Optional[Tree], trip: bool = False, stream=None):
+    """OK only in the build with device-side index checks; trip=True also makes one check fail on purpose."""
+    _check(lib.bgrpo_debug_bounds(tree.handle if tree is not None else None, int(bool(trip)), _stream(stream)), "bgrpo_debug_bounds")
 
 
 def philox_words_fill(seed, node_id, step, tag, out, n_blocks, stream=None):

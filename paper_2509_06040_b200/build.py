@@ -1,9 +1,12 @@
 """Builds libbgrpo.so (hand-written CUDA for sm_100a) in-tree with nvcc.
 
-    python -m paper_2509_06040_b200.build [--force] [--verbose]
+    python -m paper_2509_06040_b200.build [--force] [--verbose] [--debug-bounds]
 
 nvcc cross-compiles without a GPU.  Objects go to paper_2509_06040_b200/_build/,
-the shared library next to this file.
+the shared library next to this file.  --debug-bounds (or build(debug_bounds=True))
+builds libbgrpo_debug.so instead: the same sources with -DBGRPO_DEBUG_BOUNDS, in which
+every kernel checks its indices against the launch's extents (objects in _build_debug/).
+The binding loads that library when the environment has BGRPO_DEBUG_BOUNDS=1.
 """
 from __future__ import annotations
 
@@ -17,6 +20,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbgrpo.so")
+LIB_DEBUG = os.path.join(HERE, "libbgrpo_debug.so")
 SOURCES = ["api.cu", "tree_step.cu", "tree_reward.cu", "tree_fused.cu", "tree_reduce.cu", "mlp_velocity.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
@@ -36,15 +40,18 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
-        return LIB
-    os.makedirs(BUILD, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    lib = LIB_DEBUG if debug_bounds else LIB
+    objdir = BUILD + "_debug" if debug_bounds else BUILD
+    flags = NVCC_FLAGS + (["-DBGRPO_DEBUG_BOUNDS"] if debug_bounds else [])
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _deps_mtime():
+        return lib
+    os.makedirs(objdir, exist_ok=True)
     nvcc = _nvcc()
 
     def compile_one(src):
-        obj = os.path.join(BUILD, src.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        obj = os.path.join(objdir, src.replace(".cu", ".o"))
+        cmd = [nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         with open(obj + ".log", "w") as f:
             f.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
@@ -54,14 +61,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
             print(r.stderr)
         return obj
 
-    with ThreadPoolExecutor(max_workers=4) as ex:
+    with ThreadPoolExecutor(max_workers=8) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    cmd = [nvcc, "-shared", "-o", LIB, *objs, "-cudart", "static"]
+    cmd = [nvcc, "-shared", "-o", lib, *objs, "-cudart", "static"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

@@ -249,6 +249,8 @@ static void fill_step_launch(const bgrpo_tree* t, int step, const float* v_dev, 
     p->logp = t->buf.logp;
     p->table = t->buf.node_table;
     p->partialsf = t->partialsf;
+    p->status = t->status;
+    p->per_row = static_cast<int32_t>(partials_per_row(t->D));
     p->prev = t->pending;
     p->D = t->D;
     p->n_trees = t->desc.n_trees;
@@ -340,6 +342,8 @@ bgrpo_status bgrpo_tree_rollout_fused(bgrpo_tree* t, const uint8_t* split_flags_
     p.logp = t->buf.logp;
     p.table = t->buf.node_table;
     p.partialsf = t->partialsf;
+    p.status = t->status;
+    p.per_row_cap = static_cast<int32_t>(partials_per_row(t->D));
     p.D = t->D;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
@@ -409,6 +413,8 @@ static bgrpo_status reward_common(bgrpo_tree* t, const float* target, float scal
     p.r = r;
     p.partials = t->partials;
     p.counters = t->counters;
+    p.status = t->status;
+    p.nchunks_cap = t->nchunks;
     p.D = t->D;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
@@ -463,6 +469,7 @@ bgrpo_status bgrpo_tree_fusion_ess(bgrpo_tree* t, float beta, float logp_scale, 
     p.logp = t->buf.logp;
     p.ess = ess_out_dev;
     p.node_scratch = t->node_scratch;
+    p.status = t->status;
     p.lv = t->lv;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
@@ -490,6 +497,7 @@ bgrpo_status bgrpo_tree_prune(bgrpo_tree* t, int32_t width_mode, int32_t k_or_b,
     p.rbar = t->buf.rbar;
     p.table = t->buf.node_table;
     p.mask = t->buf.mask;
+    p.status = t->status;
     p.lv = t->lv;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
@@ -518,6 +526,7 @@ bgrpo_status bgrpo_tree_grpo_objective(bgrpo_tree* t, const float* logp_new_dev,
     p.mask = t->buf.mask;
     p.terms = terms_out_dev;
     p.J = J_out_dev;
+    p.status = t->status;
     p.n_trees = t->desc.n_trees;
     p.nodes_cap = t->desc.nodes_cap;
     p.nodes = t->lv.offset[t->desc.T + 1];
@@ -591,8 +600,9 @@ bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* t, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(t->status, 0, sizeof(word), as_stream(stream));
     if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
     if (e != cudaSuccess) return cuda_fail(e, "status read");
-    if (word & 4) return fail(BGRPO_ERR_CUDA, "a bounded wait inside the MLP velocity kernel ran out");
-    return (word & 1) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
+    if (word & kStatusOutOfBounds) return fail(BGRPO_ERR_CAPACITY, "a device-side index check failed and the access was skipped (debug build)");
+    if (word & kStatusWaitTimeout) return fail(BGRPO_ERR_CUDA, "a bounded wait inside the MLP velocity kernel ran out");
+    return (word & kStatusNonFinite) ? fail(BGRPO_ERR_NONFINITE, "non-finite leaf reward") : BGRPO_OK;
 }
 
 bgrpo_status bgrpo_philox_words_fill(uint64_t seed, uint32_t node_id, uint32_t step, uint32_t tag, uint32_t* out_dev, int64_t n_blocks, void* stream) {
@@ -626,10 +636,24 @@ bgrpo_status bgrpo_velocity_mlp(bgrpo_tree* t, const void* packed_dev, int32_t h
     if (!aligned(packed_dev, 1024) || !aligned(v_out_dev, 16)) return fail(BGRPO_ERR_INVALID_ARG, "misaligned buffer");
     if (t->depth >= t->desc.T) return fail(BGRPO_ERR_STATE, "tree already at depth T");
     const int i = t->depth;
-    cudaError_t e = launch_mlp(t->buf.latents, static_cast<int64_t>(t->desc.nodes_cap) * t->D, static_cast<int64_t>(t->lv.offset[i]) * t->D,
+    cudaError_t e = launch_mlp(t->buf.latents, static_cast<int64_t>(t->desc.n_trees) * t->desc.nodes_cap * t->D, static_cast<int64_t>(t->desc.nodes_cap) * t->D, static_cast<int64_t>(t->lv.offset[i]) * t->D,
                                t->desc.n_trees, static_cast<int64_t>(t->lv.width[i]) * t->desc.tokens, packed_dev, hidden,
                                v_out_dev, t->mlp_partials, t->mlp_tickets, t->status, as_stream(stream));
     return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp kernel");
+}
+
+bgrpo_status bgrpo_debug_bounds(bgrpo_tree* t, int32_t trip, void* stream) {
+#ifdef BGRPO_DEBUG_BOUNDS
+    if (trip) {
+        if (!t) return fail(BGRPO_ERR_INVALID_ARG, "tree is NULL");
+        const cudaError_t e = launch_debug_trip(t->status, as_stream(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "debug trip kernel");
+    }
+    return BGRPO_OK;
+#else
+    (void)t; (void)trip; (void)stream;
+    return fail(BGRPO_ERR_UNSUPPORTED, "this library was built without device-side index checks");
+#endif
 }
 
 void bgrpo_tree_destroy(bgrpo_tree* t) { delete t; }

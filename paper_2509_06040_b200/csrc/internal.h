@@ -118,6 +118,16 @@ struct bgrpo_tree {
     bgrpo::FinalizeDesc pending;         // level whose log-probs still have to be summed
 };
 
+// Debug build (-DBGRPO_DEBUG_BOUNDS): every kernel tests the row, chunk and element indices it derives against the
+// extents it was launched with, before the access.  A failed test sets bit 2 of the tree's status word and the access
+// is skipped; nothing traps.  bgrpo_tree_sync_status reports the word.  In the normal build the tests compile to nothing.
+#ifdef BGRPO_DEBUG_BOUNDS
+#define BGRPO_IN_BOUNDS(status, cond) ((cond) ? true : (atomicOr((status), 2), false))
+#else
+#define BGRPO_IN_BOUNDS(status, cond) true
+#endif
+constexpr int kStatusNonFinite = 1, kStatusOutOfBounds = 2, kStatusWaitTimeout = 4;
+
 namespace bgrpo {
 
 // Programmatic dependent launch: a kernel launched with launch_overlapped() may be scheduled while the kernel before it
@@ -161,6 +171,8 @@ struct StepLaunch {
     int32_t shared_noise;      // 1: finite s at a split step
     int32_t write_children;    // 1: tree_step; 0: tree_logprob (children are read, nothing but logp is written)
     float* logp_out;           // destination of the log-probs (== logp for tree_step)
+    int32_t* status;           // the tree's status word
+    int32_t per_row;           // floats reserved per node row in partialsf
     float* partialsf;          // [rows][nchunks][kStepWarps] warp sums of (z' - mean)^2
     FinalizeDesc prev;         // level to finalize in this launch's prologue (logp_out == nullptr: none)
 };
@@ -169,8 +181,8 @@ cudaError_t launch_step(const StepLaunch& p, cudaStream_t s);
 cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStream_t s);
 
 struct RewardLaunch {
-    const float* latents; const float* target; float* r; double* partials; unsigned int* counters;
-    int64_t D; int32_t n_trees, nodes_cap, nchunks, leaves, off_leaf; float scale; int32_t mode;  // 0 mse, 1 cos
+    const float* latents; const float* target; float* r; double* partials; unsigned int* counters; int32_t* status;
+    int64_t D; int32_t n_trees, nodes_cap, nchunks, nchunks_cap, leaves, off_leaf; float scale; int32_t mode;  // 0 mse, 1 cos; nchunks_cap: partial slots reserved per row
 };
 cudaError_t launch_reward(const RewardLaunch& p, cudaStream_t s);
 
@@ -184,6 +196,8 @@ struct FusedLaunch {
     float* logp;
     int32_t* table;
     float* partialsf;          // [rows][per_row]: one float per warp of the CTAs that cover a row
+    int32_t* status;           // the tree's status word
+    int32_t per_row_cap;       // floats reserved per node row in partialsf
     int64_t D;
     int32_t n_trees, nodes_cap, nchunks, per_row, T, K, shared_noise;   // nchunks: CTAs per tree
     uint32_t node_id_base;
@@ -205,19 +219,19 @@ struct FuseLaunch {
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s);
 
 struct EssLaunch {
-    const float* logp; float* ess; double* node_scratch;
+    const float* logp; float* ess; double* node_scratch; int32_t* status;
     LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes; double beta_scaled;
 };
 cudaError_t launch_fusion_ess(const EssLaunch& p, cudaStream_t s);
 
 struct PruneLaunch {
-    const float* rbar; const int32_t* table; uint8_t* mask;
+    const float* rbar; const int32_t* table; uint8_t* mask; int32_t* status;
     LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes, mode, k, last_split, ignore_last, values_in_smem; uint64_t pruned_bits;
 };
 cudaError_t launch_prune(const PruneLaunch& p, cudaStream_t s);
 
 struct ObjectiveLaunch {
-    const float* logp_new; const float* logp_old; const float* adv; const uint8_t* mask; float* terms; float* J;
+    const float* logp_new; const float* logp_old; const float* adv; const uint8_t* mask; float* terms; float* J; int32_t* status;
     int32_t n_trees, nodes_cap, nodes; double logp_scale; float clip_eps;
 };
 cudaError_t launch_objective(const ObjectiveLaunch& p, cudaStream_t s);
@@ -230,7 +244,8 @@ constexpr size_t kMlpPartialBytes = static_cast<size_t>(kMlpSplitMaxCtas) * 128 
 constexpr size_t kMlpTicketBytes = 1024;      // kMlpSplitMaxCtas counters, rounded up
 size_t mlp_packed_bytes(int hidden);
 cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, void* packed, cudaStream_t s);
-cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
+cudaError_t launch_debug_trip(int32_t* status, cudaStream_t s);     // debug build: fails one index test on purpose (no access involved)
+cudaError_t launch_mlp(const float* latents, int64_t pool_elems, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
                        const void* packed, int hidden, float* v_out, float* split_partials, unsigned int* split_tickets,
                        int32_t* status, cudaStream_t s);
 

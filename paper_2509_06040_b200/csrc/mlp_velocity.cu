@@ -284,6 +284,7 @@ __device__ __forceinline__ void convert_rows(const float* stage, unsigned char* 
 
 struct MlpArgs {
     const float* latents;     // pool base
+    int64_t pool_elems;       // elements in the pool
     int64_t tree_stride;      // elements between trees in the pool
     int64_t row_offset;       // elements from a tree's base to its frontier
     int64_t tokens_per_tree;  // frontier tokens of one tree (W_i * tokens)
@@ -467,7 +468,11 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
                 const int64_t tree = q / p.tokens_per_tree, rr = q - tree * p.tokens_per_tree;
                 int64_t seg = p.tokens_per_tree - rr;
                 if (seg > remaining) seg = remaining;
-                bulk_load(dst, p.latents + tree * p.tree_stride + p.row_offset + rr * kCh, static_cast<uint32_t>(seg) * (kCh * 4u), &sm.stage_full);
+                const int64_t first = tree * p.tree_stride + p.row_offset + rr * kCh;
+                if (!BGRPO_IN_BOUNDS(p.status, first >= 0 && first + seg * kCh <= p.pool_elems && dst + seg * kCh <= sm.stage + kTok * kCh))
+                    *abort_flag = 1;      // the copy is skipped: the tile cannot complete, so every role drains
+                else
+                    bulk_load(dst, p.latents + first, static_cast<uint32_t>(seg) * (kCh * 4u), &sm.stage_full);
                 dst += seg * kCh;
                 q += seg;
                 remaining -= seg;
@@ -662,7 +667,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
-    if (threadIdx.x == 0 && sm.abort_flag) atomicOr(p.status, 4);
+    if (threadIdx.x == 0 && sm.abort_flag) atomicOr(p.status, kStatusWaitTimeout);
 }
 
 // Reorders W1 [64][H] and W2 [H][64] (bf16 bits) into per-chunk shared-memory images: for chunk c,
@@ -695,7 +700,7 @@ cudaError_t launch_mlp_pack(const uint16_t* W1, const uint16_t* W2, int hidden, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
+cudaError_t launch_mlp(const float* latents, int64_t pool_elems, int64_t tree_stride, int64_t row_offset, int n_trees, int64_t tokens_per_tree,
                        const void* packed, int hidden, float* v_out, float* split_partials, unsigned int* split_tickets,
                        int32_t* status, cudaStream_t s) {
     static bool configured[64] = {false};
@@ -711,6 +716,7 @@ cudaError_t launch_mlp(const float* latents, int64_t tree_stride, int64_t row_of
     if (e != cudaSuccess) return e;
     MlpArgs a;
     a.latents = latents;
+    a.pool_elems = pool_elems;
     a.tree_stride = tree_stride;
     a.row_offset = row_offset;
     a.tokens_per_tree = tokens_per_tree;

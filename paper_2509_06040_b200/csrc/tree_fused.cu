@@ -35,6 +35,8 @@ __device__ __forceinline__ void emit_child(const FusedLaunch& p, const Ctx& cx, 
                                            int split_step, int branch_id, float g, const float4 (&m)[kFusedVec],
                                            const float4 (&xi0)[kFusedVec], bool shared, float4 (&c)[kFusedVec]) {
     const uint32_t gid = cx.gid0 + static_cast<uint32_t>(child_local);
+    if (!BGRPO_IN_BOUNDS(p.status, child_local > 0 && child_local < p.nodes_cap && parent_local >= 0 && parent_local < child_local &&
+                                       (cx.chunk + 1) * (kFusedThreads / 32) <= p.per_row_cap)) return;
     float acc = 0.0f;
     float4* row = cx.tree_base + static_cast<size_t>(child_local) * static_cast<size_t>(p.D >> 2);
 #pragma unroll
@@ -162,6 +164,7 @@ finalize_tree_kernel(const __grid_constant__ FusedLaunch p, int32_t nodes) {
     while (step + 1 < p.T && local >= p.off[step + 2]) ++step;
     const int64_t row = static_cast<int64_t>(tree) * p.nodes_cap + local;
     const int per_row = p.per_row;
+    if (!BGRPO_IN_BOUNDS(p.status, local < p.nodes_cap && per_row <= p.per_row_cap)) return;
     const float* q = p.partialsf + row * per_row;
     double s = 0.0;
     for (int c = lane; c < per_row; c += 32) s += static_cast<double>(__ldcg(q + c));

@@ -54,6 +54,7 @@ fuse_advantage_kernel(const FuseLaunch p) {
         const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
         for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads) {
             const int c0 = offc + j * fan;
+            if (!BGRPO_IN_BOUNDS(p.status, off + j < offc && c0 + fan <= p.nodes && p.nodes <= p.nodes_cap)) continue;
             if (fan == 1) {      // an only child: its value is the parent's, and log S just picks up the edge
                 rb[off + j] = rb[c0];
                 ls[off + j] = (la ? la[c0] : beta * static_cast<double>(p.logp[row0 + c0])) + ls[c0];
@@ -127,6 +128,7 @@ fusion_ess_kernel(const EssLaunch p) {
         const int off = p.lv.offset[d], offc = p.lv.offset[d + 1];
         for (int j = threadIdx.x; j < p.lv.width[d]; j += kTreeThreads) {
             const int c0 = offc + j * fan;
+            if (!BGRPO_IN_BOUNDS(p.status, off + j < offc && c0 + fan <= p.nodes && p.nodes <= p.nodes_cap)) continue;
             double a1[BGRPO_MAX_K], a2[BGRPO_MAX_K];
             double m1 = -INFINITY, m2 = -INFINITY;
 #pragma unroll
@@ -239,6 +241,7 @@ prune_kernel(const PruneLaunch p) {
             if (extreme_key(v, static_cast<uint32_t>(l), false) >= best_cut || extreme_key(v, static_cast<uint32_t>(l), true) >= worst_cut) {
                 int n = off + l;
                 for (int guard = 0; n >= 0 && guard <= T; ++guard) {       // root path through the node table
+                    if (!BGRPO_IN_BOUNDS(p.status, n < p.nodes)) break;
                     keep[n] = 1;
                     n = p.table[row0 + n];
                 }
@@ -273,6 +276,7 @@ prune_kernel(const PruneLaunch p) {
                                             (p.mode == BGRPO_WIDTH_LAST_SPLIT_TOPK && e - 1 == p.last_split));
             if (ranked) {
                 const int sib0 = s_off[e] + pj * fan;
+                if (!BGRPO_IN_BOUNDS(p.status, sib0 >= 0 && sib0 + fan <= p.nodes)) break;
                 const float v = rbar[sib0 + b];
                 int rank = 0;
                 for (int q = 0; q < fan; ++q) rank += beats(rbar[sib0 + q], q, v, b) ? 1 : 0;
@@ -293,6 +297,7 @@ objective_kernel(const ObjectiveLaunch p) {
     const int64_t row0 = static_cast<int64_t>(tree) * p.nodes_cap;
     double sum = 0.0;
     int cnt = 0;
+    if (!BGRPO_IN_BOUNDS(p.status, p.nodes <= p.nodes_cap && tree < p.n_trees)) return;
     for (int n = threadIdx.x; n < p.nodes; n += kTreeThreads) {
         float term = 0.0f;
         if (n > 0 && p.mask[row0 + n]) {

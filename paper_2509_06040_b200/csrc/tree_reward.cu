@@ -116,6 +116,7 @@ reward_kernel(const __grid_constant__ RewardLaunch p) {
     const float4* __restrict__ tg = reinterpret_cast<const float4*>(p.target + static_cast<int64_t>(tree) * p.D);
     constexpr int NV = (MODE == 0) ? 1 : 3;
     const uint32_t c0 = static_cast<uint32_t>(chunk) * kRewardChunkVec;
+    if (!BGRPO_IN_BOUNDS(p.status, tree < p.n_trees && p.off_leaf + l < p.nodes_cap && c0 < D4 && p.nchunks <= p.nchunks_cap)) return;
     double dsum[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) dsum[v] = 0.0;
@@ -149,6 +150,7 @@ reward_finish_kernel(const __grid_constant__ RewardLaunch p) {
     if (row >= p.n_trees * p.leaves) return;
     const int tree = row / p.leaves;
     const int64_t node_row = static_cast<int64_t>(tree) * p.nodes_cap + p.off_leaf + (row - tree * p.leaves);
+    if (!BGRPO_IN_BOUNDS(p.status, p.off_leaf + p.leaves <= p.nodes_cap && p.nchunks <= p.nchunks_cap)) return;
     if (MODE == 0) {
         const double ss = row_total(p.partials, node_row, 0, p.nchunks);
         if ((threadIdx.x & 31) == 0) p.r[row] = static_cast<float>(-ss / static_cast<double>(p.D));

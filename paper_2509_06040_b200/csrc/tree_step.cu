@@ -29,6 +29,7 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
     const int chunk = blockIdx.x % nchunks;
     const int tree = blockIdx.x / nchunks;
     const int64_t D4 = D >> 2;
+    if (!BGRPO_IN_BOUNDS(status, tree < n_trees && static_cast<int64_t>(chunk) * kChunkVec < D4)) return;
     float4* z = reinterpret_cast<float4*>(latents + static_cast<int64_t>(tree) * nodes_cap * D);
     const uint32_t gid = node_id_base + static_cast<uint32_t>(tree) * nodes_cap;
 #pragma unroll
@@ -72,13 +73,14 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
 // Adds up the pending level's partial sums: one warp per row, lanes stride over the row's nchunks * kStepWarps floats
 // in index order, then a fixed shuffle tree; double throughout.
 __device__ __forceinline__ void finalize_rows(const FinalizeDesc& f, const float* partialsf, int32_t n_trees, int32_t nodes_cap,
-                                              int32_t nchunks, int64_t D, int warp_global, int warps_total) {
+                                              int32_t nchunks, int64_t D, int warp_global, int warps_total, int32_t* status, int32_t per_row_cap) {
     const int lane = threadIdx.x & 31;
     const int n_rows = n_trees * f.W;
     const int per_row = nchunks * kStepWarps;
     for (int idx = warp_global; idx < n_rows; idx += warps_total) {
         const int tree = idx / f.W;
         const int64_t row = static_cast<int64_t>(tree) * nodes_cap + f.off + (idx - tree * f.W);
+        if (!BGRPO_IN_BOUNDS(status, f.off + f.W <= nodes_cap && per_row <= per_row_cap)) continue;
         const float* q = partialsf + row * per_row;
         double s = 0.0;
         for (int c = lane; c < per_row; c += 32) s += static_cast<double>(__ldcg(q + c));
@@ -171,7 +173,7 @@ step_kernel(const __grid_constant__ StepLaunch p) {
     pdl_wait();           // the parents, the velocity and the pending partial sums come from earlier kernels
     // the previous level's log-probs (a handful of rows): summed by this launch
     if (p.prev.logp_out != nullptr)
-        finalize_rows(p.prev, p.partialsf, p.n_trees, p.nodes_cap, p.nchunks, p.D, blockIdx.x * kStepWarps + warp, gridDim.x * kStepWarps);
+        finalize_rows(p.prev, p.partialsf, p.n_trees, p.nodes_cap, p.nchunks, p.D, blockIdx.x * kStepWarps + warp, gridDim.x * kStepWarps, p.status, p.per_row);
 
     const int chunk = blockIdx.x % p.nchunks;
     const int row = blockIdx.x / p.nchunks;             // tree * W_in + j
@@ -184,6 +186,8 @@ step_kernel(const __grid_constant__ StepLaunch p) {
     const int parent = p.off_in + j;
     const int child0 = p.off_out + j * FAN;
     const bool streamed = (p.v != nullptr);
+    if (!BGRPO_IN_BOUNDS(p.status, tree < p.n_trees && parent < p.nodes_cap && child0 + FAN <= p.nodes_cap && e_base < D4 &&
+                                       (chunk + 1) * kStepWarps <= p.per_row)) return;
     const float4* __restrict__ zp = reinterpret_cast<const float4*>(p.latents + (tree_row0 + parent) * p.D) + e_base;
     const float4* __restrict__ xop = (streamed ? reinterpret_cast<const float4*>(p.v + static_cast<int64_t>(row) * p.D)
                                                : reinterpret_cast<const float4*>(p.mu + static_cast<int64_t>(tree) * p.D)) + e_base;
@@ -225,11 +229,12 @@ step_kernel(const __grid_constant__ StepLaunch p) {
 
 // Flush: adds up a pending level outside a step launch (the tree is complete, or tree_logprob is done).
 __global__ void __launch_bounds__(kStreamThreads)
-finalize_kernel(const FinalizeDesc f, const float* partialsf, int32_t n_trees, int32_t nodes_cap, int32_t nchunks, int64_t D) {
+finalize_kernel(const FinalizeDesc f, const float* partialsf, int32_t n_trees, int32_t nodes_cap, int32_t nchunks, int64_t D,
+                int32_t* status, int32_t per_row_cap) {
     pdl_release();
     pdl_wait();
     finalize_rows(f, partialsf, n_trees, nodes_cap, nchunks, D, blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5),
-                  gridDim.x * (kStreamThreads / 32));
+                  gridDim.x * (kStreamThreads / 32), status, per_row_cap);
 }
 
 __global__ void philox_words_kernel(const __grid_constant__ PhiloxKeys keys, uint32_t node, uint32_t step, uint32_t tag, uint4* out, int64_t nblk) {
@@ -241,6 +246,10 @@ __global__ void philox_normals_kernel(const __grid_constant__ PhiloxKeys keys, u
     if (i < nblk) out[i] = noise4(static_cast<uint32_t>(i), node, step, tag, keys);
 }
 
+__global__ void debug_trip_kernel(int32_t* status) {
+    if (!BGRPO_IN_BOUNDS(status, threadIdx.x > 0)) return;      // thread 0 fails the test; nothing is accessed
+}
+
 template <int FAN>
 cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t s) {
     if (!p.write_children) return launch_overlapped(step_kernel<FAN, false, false>, grid, kStepThreads, 0, s, p);
@@ -249,6 +258,11 @@ cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t
 }
 
 }  // namespace
+
+cudaError_t launch_debug_trip(int32_t* status, cudaStream_t s) {
+    debug_trip_kernel<<<1, 32, 0, s>>>(status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_root(const bgrpo_tree* t, cudaStream_t s) {
     const unsigned int grid = static_cast<unsigned int>(t->desc.n_trees) * t->nchunks;
@@ -274,7 +288,8 @@ cudaError_t launch_finalize(const bgrpo_tree* t, const FinalizeDesc& f, cudaStre
     const int rows = t->desc.n_trees * f.W;
     const int grid = (rows + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
     return launch_overlapped(finalize_kernel, grid < 1 ? 1 : grid, kStreamThreads, 0, s, f, static_cast<const float*>(t->partialsf),
-                             t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D);
+                             t->desc.n_trees, t->desc.nodes_cap, t->nchunks_step, t->D, t->status,
+                             static_cast<int32_t>(partials_per_row(t->D)));
 }
 
 cudaError_t launch_philox_words(uint64_t seed, uint32_t node, uint32_t step, uint32_t tag, uint32_t* out, int64_t nblk, cudaStream_t s) {
