@@ -133,6 +133,11 @@ bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* tree, const float* mu_dev, f
  * bound linear velocity.  One fused kernel appends the children's node-table rows, writes their latents and the
  * partial sums of the per-element-mean Gaussian log-prob of each new edge,
  *   logp = -(1/D) sum_e (z'_e - mu_e)^2 / (2 g_i^2) - ln g_i - 0.5 ln(2 pi)      (multiply by D for the joint density).
+ * The value is stored as float32: its rounding (about 1e-7 at |logp| ~ 1) is multiplied by whatever scale a caller
+ * applies later, so logp_scale = D in tree_fuse_advantage / tree_grpo_objective gives joint densities good to about
+ * 1e-7 * D in the exponent - fine for D up to a few thousand, meaningless at D ~ 1e5 (use a scale of order 1 there, as the
+ * workloads do).  At step time the squared residual is taken as g^2 xi^2 from the drawn noise, tree_logprob takes it
+ * from the stored child; the two agree to the rounding of the child (test: rho = 1 within 1e-5).
  * The sums are completed, in a fixed order, by the next call for this tree that is enqueued on the stream (the next
  * tree_step's kernel does it in its prologue) and at the latest by the step that completes the tree, which enqueues a
  * small flush kernel: buffers.logp of a level is final once one of those has run.  Use one stream per tree handle.
@@ -140,7 +145,8 @@ bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* tree, const float* mu_dev, f
 bgrpo_status bgrpo_tree_step(bgrpo_tree* tree, int32_t split_flag, const float* v_dev, void* stream);
 
 /* tree_rollout_fused: all T steps of tree_step in one launch, for the bound closed-form velocity (Branch Rollout
- * Algorithm: "reusing shared prefixes"; Eq. 2; Algorithm 1 "Build rollout tree").  That velocity acts on every latent
+ * Algorithm, where a prefix is computed once for all the leaves below it; Eq. 2; Algorithm 1 "Build rollout tree").
+ * That velocity acts on every latent
  * element by itself, so one thread can carry its elements from the root to every leaf, depth first, and write each
  * node once: nothing is read back between depths.  Call it on a freshly initialised or reset tree.  split_flags_host:
  * host array of T flags, non-zero = step i forks every node into K children.  Latents, node table and log-probs are the
@@ -193,8 +199,8 @@ bgrpo_status bgrpo_tree_fuse_advantage(bgrpo_tree* tree, const float* leaf_rewar
  * ess_out_dev: device [n_trees][nodes_cap] float32. */
 bgrpo_status bgrpo_tree_fusion_ess(bgrpo_tree* tree, float beta, float logp_scale, float* ess_out_dev, void* stream);
 
-/* tree_prune: gradient mask per node-step; reads buffers.rbar, writes buffers.mask only ("pruning ... affects
- * backpropagation but not forward rollouts or reward evaluation").  mask(n) = keep_width(n) AND step(depth(n)-1) not in
+/* tree_prune: gradient mask per node-step; reads buffers.rbar, writes buffers.mask only (section "Pruning Strategies":
+ * pruning selects what is back-propagated and leaves rollouts, rewards and advantages as they are).  mask(n) = keep_width(n) AND step(depth(n)-1) not in
  * pruned_steps AND n is not the root AND (ignore_last_step == 0 OR depth(n) < T).  Width ranking compares the float32
  * rbar values, ties to the lower branch (or leaf) index; a pruned child masks its whole subtree.
  * pruned_steps_host: host array of n_pruned steps in 0..T-1 (the set D of "Depth Pruning"), may be NULL if 0. */
@@ -211,8 +217,8 @@ bgrpo_status bgrpo_tree_prune(bgrpo_tree* tree, int32_t width_mode, int32_t k_or
 bgrpo_status bgrpo_tree_grpo_objective(bgrpo_tree* tree, const float* logp_new_dev, const float* logp_old_dev, float logp_scale,
                                        float clip_eps, float* terms_out_dev, float* J_out_dev, void* stream);
 
-/* Hybrid ODE-SDE schedule (ablation "Hybrid ODE-SDE": all branching steps are preserved as SDE, a sliding window determines
- * additional SDE steps, the remaining updates are ODE steps).  sde_flags_host: host array of T bytes, 1 = step i is
+/* Hybrid ODE-SDE schedule (ablation "Hybrid ODE-SDE": split steps stay stochastic, a sliding window names further
+ * stochastic steps, every other step is deterministic).  sde_flags_host: host array of T bytes, 1 = step i is
  * stochastic, 0 = deterministic (sigma = 0 for that step: drift -v only, no noise drawn, log-prob written as 0, and
  * tree_prune masks its node-steps); NULL restores "every step is SDE".  Host only; affects the steps taken afterwards.
  * A later tree_step with split_flag != 0 on an ODE step returns INVALID_ARG (identical children carry no signal). */
@@ -222,8 +228,8 @@ bgrpo_status bgrpo_tree_set_sde_steps(bgrpo_tree* tree, const uint8_t* sde_flags
 bgrpo_status bgrpo_mix_sde_steps(int32_t T, const int32_t* split_steps, int32_t n_splits, int32_t iter, int32_t window,
                                  int32_t every, int32_t start, uint8_t* flags_out);
 
-/* Sliding-window schedule of depth pruning (ablation "Pruning Strategies": window initialised at the last split point,
- * size 4, one step deeper every 30 iterations, until a stop depth): steps_out[j] = min(start + iter/every, stop-size) + j.
+/* Sliding-window schedule of depth pruning (ablation "Pruning Strategies": the window starts at the last split step,
+ * spans four steps and moves one step deeper every thirty iterations, up to a stop depth): steps_out[j] = min(start + iter/every, stop-size) + j.
  * stop < 0 = no stop.  Host only; steps_out holds `size` entries. */
 bgrpo_status bgrpo_depth_window(int32_t iter, int32_t start, int32_t size, int32_t every, int32_t stop,
                                 int32_t* steps_out, int32_t* n_out);

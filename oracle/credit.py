@@ -7,17 +7,17 @@ Readings where the paper is silent
 * N_d of Eq. 4 is the set of depth-d nodes of ONE prompt's tree; sigma_d is the
   population standard deviation, so a depth with a single node gets A = 0.
 * The root has no incoming edge: its advantage is 0 and its mask is 0.
-* Width pruning has three modes: top-k children at every split
-  ("retain only the locally better child at each branch", ablation text), top-k
-  children at the last split only ("Parent-Top1 ... at the last branching step",
-  method text) and Extreme-b (best b and worst b leaves).  A pruned child loses
+* Width pruning has three modes: top-k children at every split (the ablation's
+  reading of Parent-Top1), top-k children at the last split only (the method
+  section's reading, "Width Pruning") and Extreme-b (best b and worst b leaves).
+  A pruned child loses
   its incoming edge and its whole subtree; ancestors it shares with kept
   children stay.  Ties rank the lower branch index (or leaf index) first.
 * Depth pruning is indexed by step: step i in the pruned set removes the edges
   i -> i+1, i.e. the nodes of depth i+1.
-* The sliding window of the ablation text ("initialized at the last split point,
-  size 4, shifts by one denoising step every 30 training iterations" until a stop
-  depth) gives steps min(start + iter // every, stop - size) + 0..size-1.
+* The sliding window of the ablation "Pruning Strategies" (it starts at the last
+  split step, spans four steps and moves one step deeper every thirty iterations,
+  up to a stop depth) gives steps min(start + iter // every, stop - size) + 0..size-1.
 """
 from __future__ import annotations
 

@@ -3,14 +3,14 @@
     python paper_2509_06040_b200/csrc/gelu_poly_fit.py
 
 2 GELU(x) = x + x erf(x / sqrt 2) = x + s Q(s), s = x^2.  Q (degree 2 in s) is fitted to erf(x / sqrt 2) / x on
-|x| <= 1.5 so that the largest error of s Q(s) is smallest (weighted least squares with Lawson's reweighting); the
+|x| <= 1 so that the largest error of s Q(s) is smallest (weighted least squares with Lawson's reweighting); the
 kernel evaluates in bf16, so the coefficients are rounded to bf16 one after the other, each time refitting the ones
 not yet fixed.  Prints the coefficients, their bf16 bit patterns and the largest error of the rounded polynomial.
 """
 import numpy as np
 from scipy.special import erf
 
-RANGE, DEGREE = 1.5, 2
+RANGE, DEGREE = 1.0, 2
 
 
 def to_bf16(x):

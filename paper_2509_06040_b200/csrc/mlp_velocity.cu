@@ -241,18 +241,18 @@ __device__ __forceinline__ uint32_t bf2_fma(uint32_t a, uint32_t b, uint32_t c) 
     asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
-// Twice the erf-form GELU for |x| < 1.5 without a special-function instruction:
+// Twice the erf-form GELU for |x| < 1 without a special-function instruction:
 //     2 GELU(x) = x + x erf(x / sqrt 2) = x + s Q(s),   s = x^2,
-// with Q a quadratic in s fitted to erf(x / sqrt 2) / x on [0, 1.5] (minimax in s Q(s), the coefficients rounded to bf16
-// one after the other and the rest refitted by csrc/gelu_poly_fit.py; the polynomial is within 6.3e-4 of the function).
+// with Q a quadratic in s fitted to erf(x / sqrt 2) / x on [0, 1] (minimax in s Q(s), the coefficients rounded to bf16
+// one after the other and the rest refitted by csrc/gelu_poly_fit.py; the polynomial is within 8e-5 of the function).
 // Evaluated on a packed pair in bf16: one multiply and three fused multiply-adds on the FMA pipe, where one hardware
 // tanh per activation (sixteen per clock and SM) bounds the whole stage at twice the tensor-core time.  The last
 // operation, fma(t, s, x), adds the small even part to x and rounds once, so for the usual |x| << 1 the result differs
 // from the correctly rounded activation by the rounding of x to bf16 and little else.
-constexpr uint32_t kGeluQ0 = 0x3f4b3f4bu;   //  0.79296875
-constexpr uint32_t kGeluQ1 = 0xbdf8bdf8u;   // -0.12109375
-constexpr uint32_t kGeluQ2 = 0x3c383c38u;   //  0.01123046875
-constexpr uint32_t kGeluRangeBf16 = 0x3fc0u;   // bf16 bits of 1.5: the polynomial's range
+constexpr uint32_t kGeluQ0 = 0x3f4c3f4cu;   //  0.796875
+constexpr uint32_t kGeluQ1 = 0xbe04be04u;   // -0.12890625
+constexpr uint32_t kGeluQ2 = 0x3c723c72u;   //  0.0147705078125
+constexpr uint32_t kGeluRangeBf16 = 0x3f80u;   // bf16 bits of 1.0: the polynomial's range
 __device__ __forceinline__ uint32_t gelu_x2_poly(uint32_t xb) {
     const uint32_t s = bf2_mul(xb, xb);
     uint32_t t = bf2_fma(kGeluQ2, s, kGeluQ1);
@@ -605,7 +605,7 @@ mlp_velocity_kernel(const __grid_constant__ MlpArgs p) {
         // 32 accumulator columns -> 16 registers of packed bf16 activation pairs
         // One chunk of this warp: 64 accumulator columns arrive as float32, are rounded to packed bf16 pairs at once (32
         // registers) and D1 is handed back before any arithmetic, so GEMM1 of chunk g + 2 runs under the activation of
-        // chunk g.  The packed polynomial covers |x| < 1.5; a running maximum of magnitudes shows whether any of this
+        // chunk g.  The packed polynomial covers |x| < 1; a running maximum of magnitudes shows whether any of this
         // thread's 64 values lies outside (or is not finite), and only then the thread takes the hardware-tanh form
         // for its values.  With weights and latents of the usual scale (pre-activations of standard deviation ~0.2) that
         // never happens.

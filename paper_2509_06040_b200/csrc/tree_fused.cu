@@ -2,8 +2,8 @@
 // Gaussian-target velocity).  With such a velocity an element's trajectory through the tree never looks at any other
 // element, so a thread can carry its elements from the root through every depth in registers, depth first, and
 // write each node's latent exactly once: the parent read of the level-by-level step kernel disappears (4 bytes per
-// element and node-step instead of 8) and the T launches become one.  "Shared prefixes amortize computation"
-// (Branch Rollout Algorithm) is taken literally: a prefix is computed once and never re-read.
+// element and node-step instead of 8) and the T launches become one.  The saving the Branch Rollout Algorithm draws
+// from shared prefixes is taken literally: a prefix is computed once and never re-read.
 //
 // Every node gets exactly the value the level-by-level path gives it: the same Philox counters (element block, global
 // node id, step, tag), the same float32 expressions (mean = ca z + cb mu, child = g xi + mean, Eq. 2 noise mixing).

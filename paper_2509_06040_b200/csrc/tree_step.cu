@@ -109,13 +109,17 @@ template <int FAN, bool SHARED, bool WRITE, bool FULL>
 __device__ __forceinline__ void compute_tile(const StepLaunch& p, const float4 (&z)[kStepVec], const float4 (&x)[kStepVec],
                                              uint32_t vecs, uint32_t e_base, uint32_t D4, float4* zc, uint32_t gid_parent,
                                              uint32_t gid_child0, float (&acc)[FAN]) {
+    const bool noisy = p.g != 0.0f;
 #pragma unroll
     for (int k = 0; k < kStepVec; ++k) {
         const uint32_t t = threadIdx.x + k * kStepThreads;
         if (FULL || t < vecs) {
             const uint32_t e = e_base + t;
             float4 xi[FAN];
-            if (WRITE) {
+            if (WRITE && !noisy) {       // deterministic step (sigma = 0): no noise is drawn, the child is the mean
+#pragma unroll
+                for (int b = 0; b < FAN; ++b) xi[b] = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else if (WRITE) {
                 float4 xi0 = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (SHARED) xi0 = noise4(e, gid_parent, p.step, BGRPO_TAG_SHARED, p.keys);
 #pragma unroll

@@ -99,7 +99,11 @@ def test_mlp_stage_full_size_sampled(B, name, depth):
     ref = mlp.mlp_velocity(zt[idx], inp.W1, inp.W2)
     out = got[torch.from_numpy(idx).cuda()].cpu().numpy()
     rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
-    assert np.all(np.abs(out - ref) <= 2e-2 * np.abs(ref) + 2e-2 * rms), float(np.abs(out - ref).max() / rms)
+    d = np.abs(out - ref)
+    print(f"{name} depth {depth}: worst |d|/rms(v) = {d.max() / rms:.4f}, rms |d|/rms(v) = {np.sqrt(np.mean(d ** 2)) / rms:.4f}")
+    assert np.all(d <= 2e-2 * np.abs(ref) + 2e-2 * rms), float(d.max() / rms)
+    large = np.abs(ref) >= rms
+    assert np.all(d[large] <= 2e-2 * np.abs(ref[large]))      # plain relative bound where the output is not small
     assert not torch.isnan(got).any()            # every token of the frontier was written
 
 
