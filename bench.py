@@ -297,8 +297,8 @@ def _noop(_):
     return 0
 
 
-ORACLE_SAMPLE = {   # (single-thread fraction, all-cores fraction) of one tree's latent row
-    "toy": (1.0, 1.0), "image": (0.05, 0.4), "image_batch": (0.05, 0.4), "group": (0.01, 0.08), "video": (0.25, 1.0)}
+ORACLE_SAMPLE = {   # (single-thread fraction, all-cores fraction) of one tree's latent row: about 10 s of CPU work each
+    "toy": (1.0, 1.0), "image": (0.15, 1.0), "image_batch": (0.15, 1.0), "group": (0.05, 0.3), "video": (0.5, 1.0)}
 
 
 def host_cores():
@@ -414,8 +414,7 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
                  "frac": r4(gbs / hbm_peak), "frac_of_nominal_8TBs": r4(gbs / NOMINAL_HBM_GBS), "peak_source": peaks["_source"],
                  "basis": basis, "launches_per_pass": w.T, "ms_per_pass": r4(t_step.sum()),
                  "all_launches_gbs": r4(sb.sum() / (t_step.sum() * 1e-3) / 1e9),
-                 "widest_launch": {"step": widest, "bytes": float(sb[widest]), "ms": r4(t_step[widest]),
-                                   "gbs": r4(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
+                 "widest_launch": {"step": widest, "ms": r4(t_step[widest]), "gbs": r4(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
                  "traffic": r4(ncu_traffic("step_kernel", float(sum(c * w.D for c in step_children(w))) / w.T))}
     if w.velocity == "linear":
         # With the closed-form velocity the T step launches follow one another with nothing in between.  Between one pair
@@ -436,7 +435,7 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
             tot += g0.elapsed_time(g1)
         ms_group = tot / reps
         roof_step["algorithmic_gbs_l2_assisted"] = {"gbs": r4(sb[:-1].sum() / (ms_group * 1e-3) / 1e9), "ms": r4(ms_group),
-                                                    "launches": w.T - 1, "bytes": float(sb[:-1].sum())}
+                                                    "launches": w.T - 1}
     reward_bytes = 0.0 if w.reward == "mixture" else float(w.n_trees * (w.leaves + 1) * 4 * w.D)   # leaf rows once, target once per tree
     parts = {"mlp": t_mlp.sum(), "step": t_step.sum(), "root": t_root, "leaf_reward": t_tail[0], "fuse_advantage": t_tail[1],
              "prune": t_tail[2]}
@@ -753,8 +752,7 @@ def run_ours(args, w):
                        "rollout": rollout_kind, "parallelism": f"dp{world} over trees, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": r4(e2e_value), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "mode": "inputs of pass k+1 copied on a second stream under pass k",
-                    "one_pass_at_a_time": r4(e2e_serial)},
+                    "mode": "next pass's inputs copied under this pass", "one_pass_at_a_time": r4(e2e_serial)},
             "gpu_launches": launches, "clocks": clocks, "kernel_ms_per_pass": breakdown, "savings": savings, "also": also,
         }
         if roof is not roof_step:

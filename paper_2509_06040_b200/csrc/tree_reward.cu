@@ -101,8 +101,11 @@ __device__ __forceinline__ void accumulate_chunk(const float4* __restrict__ z, c
     }
 }
 
+// Three or four CTAs per SM: with that many registers to spend the compiler keeps a batch's loads ahead of its
+// arithmetic (left to aim at full occupancy it sinks every load to its first use, and the kernel waits on one 128-bit load
+// at a time; measured 70.7 us at full occupancy against 54.3 us here on 512 rows of 129 600 elements).
 template <int MODE>
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, MODE == 0 ? 3 : 4)
 reward_kernel(const __grid_constant__ RewardLaunch p) {
     pdl_release();
     pdl_wait();

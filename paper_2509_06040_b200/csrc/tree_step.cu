@@ -68,7 +68,8 @@ root_kernel(float* latents, int32_t* table, float* logp, unsigned int* counters,
 //
 // FAN children per parent; SHARED: xi_b mixes a per-parent xi_0 (finite s at a split step); WRITE: true =
 // tree_step (draw noise, write children), false = tree_logprob (read children, score them); FULL: the tile holds
-// kStepChunkVec float4, so no element needs a bounds test.
+// kStepChunkVec float4, so no element needs a bounds test; NOISY = false: a deterministic step (sigma = 0) of the
+// hybrid schedule, no noise is generated at all.
 
 // Adds up the pending level's partial sums: one warp per row, lanes stride over the row's nchunks * kStepWarps floats
 // in index order, then a fixed shuffle tree; double throughout.
@@ -105,18 +106,17 @@ __device__ __forceinline__ void load_tile(const float4* __restrict__ zp, const f
     }
 }
 
-template <int FAN, bool SHARED, bool WRITE, bool FULL>
+template <int FAN, bool SHARED, bool WRITE, bool FULL, bool NOISY>
 __device__ __forceinline__ void compute_tile(const StepLaunch& p, const float4 (&z)[kStepVec], const float4 (&x)[kStepVec],
                                              uint32_t vecs, uint32_t e_base, uint32_t D4, float4* zc, uint32_t gid_parent,
                                              uint32_t gid_child0, float (&acc)[FAN]) {
-    const bool noisy = p.g != 0.0f;
 #pragma unroll
     for (int k = 0; k < kStepVec; ++k) {
         const uint32_t t = threadIdx.x + k * kStepThreads;
         if (FULL || t < vecs) {
             const uint32_t e = e_base + t;
             float4 xi[FAN];
-            if (WRITE && !noisy) {       // deterministic step (sigma = 0): no noise is drawn, the child is the mean
+            if (WRITE && !NOISY) {       // deterministic step (sigma = 0): no noise is drawn, the child is the mean
 #pragma unroll
                 for (int b = 0; b < FAN; ++b) xi[b] = make_float4(0.f, 0.f, 0.f, 0.f);
             } else if (WRITE) {
@@ -169,7 +169,7 @@ __device__ __forceinline__ void compute_tile(const StepLaunch& p, const float4 (
     }
 }
 
-template <int FAN, bool SHARED, bool WRITE>
+template <int FAN, bool SHARED, bool WRITE, bool NOISY = true>
 __global__ void __launch_bounds__(kStepThreads, kStepCtasPerSm)
 step_kernel(const __grid_constant__ StepLaunch p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -205,10 +205,10 @@ step_kernel(const __grid_constant__ StepLaunch p) {
     float4 z[kStepVec], x[kStepVec];
     if (vecs == kStepChunkVec) {
         load_tile<true>(zp, xop, streamed, vecs, z, x);
-        compute_tile<FAN, SHARED, WRITE, true>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
+        compute_tile<FAN, SHARED, WRITE, true, NOISY>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
     } else {
         load_tile<false>(zp, xop, streamed, vecs, z, x);
-        compute_tile<FAN, SHARED, WRITE, false>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
+        compute_tile<FAN, SHARED, WRITE, false, NOISY>(p, z, x, vecs, e_base, D4, zc, gid_parent, gid_child0, acc);
     }
     // one float per (child row, chunk, warp); summed later in a fixed order
 #pragma unroll
@@ -257,6 +257,7 @@ __global__ void debug_trip_kernel(int32_t* status) {
 template <int FAN>
 cudaError_t launch_step_fan(const StepLaunch& p, unsigned int grid, cudaStream_t s) {
     if (!p.write_children) return launch_overlapped(step_kernel<FAN, false, false>, grid, kStepThreads, 0, s, p);
+    if (p.g == 0.0f) return launch_overlapped(step_kernel<FAN, false, true, false>, grid, kStepThreads, 0, s, p);     // ODE step
     if (p.shared_noise) return launch_overlapped(step_kernel<FAN, true, true>, grid, kStepThreads, 0, s, p);
     return launch_overlapped(step_kernel<FAN, false, true>, grid, kStepThreads, 0, s, p);
 }
