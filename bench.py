@@ -46,12 +46,15 @@ NOMINAL_HBM_GBS = 8000.0
 # per launch is bytes-per-unit times the units of an average launch of the timed workload (traffic grows in
 # proportion to the units).  It is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {
-    "step_kernel": {"bytes": 75.599616e6 + 12.611840e6, "units": 8 * 2096640,
-                    "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "0f5299a50f5b"},
-    "mlp_velocity_kernel": {"bytes": 266.272e6 + 217.108224e6, "units": 1036800,
-                            "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "unset"},
-    "rollout_fused_kernel": {"bytes": 16.817152e6 + 866.026752e6, "units": 110 * 2096640,
-                             "sources": ("tree_fused.cu", "philox.cuh"), "shape": "kFused", "source_hash": "b6671b3e66cb"},
+    # step kernel: one capture per operand layout (8 B/element with the closed-form velocity, 12 B/element with a velocity buffer)
+    "step_kernel_linear": {"bytes": 75.596544e6 + 13.034496e6, "units": 8 * 2096640,             # profiles/step_kernel_video.md
+                           "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d569995ada83"},
+    "step_kernel_mlp": {"bytes": 531.169024e6 + 215.974400e6, "units": 32 * 16 * 129600,         # profiles/step_kernel_image_batch.md
+                        "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d569995ada83"},
+    "mlp_velocity_kernel": {"bytes": 266.334720e6 + 215.852032e6, "units": 1036800,       # profiles/mlp_velocity_kernel_image_batch.md
+                            "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "dce4af837ea0"},
+    "rollout_fused_kernel": {"bytes": 16.816640e6 + 866.172416e6, "units": 110 * 2096640,  # profiles/rollout_fused_kernel_video.md
+                             "sources": ("tree_fused.cu", "philox.cuh"), "shape": "kFused", "source_hash": "d4f0707c5632"},
 }
 
 
@@ -415,7 +418,7 @@ def kernel_rooflines(s, w, peaks, flush_buf, reps):
                  "basis": basis, "launches_per_pass": w.T, "ms_per_pass": r4(t_step.sum()),
                  "all_launches_gbs": r4(sb.sum() / (t_step.sum() * 1e-3) / 1e9),
                  "widest_launch": {"step": widest, "ms": r4(t_step[widest]), "gbs": r4(sb[widest] / (t_step[widest] * 1e-3) / 1e9)},
-                 "traffic": r4(ncu_traffic("step_kernel", float(sum(c * w.D for c in step_children(w))) / w.T))}
+                 "traffic": r4(ncu_traffic("step_kernel_" + w.velocity, float(sum(c * w.D for c in step_children(w))) / w.T))}
     if w.velocity == "linear":
         # With the closed-form velocity the T step launches follow one another with nothing in between.  Between one pair
         # of events a launch's ramp overlaps its predecessor's tail and the level just written is still in the L2 when the

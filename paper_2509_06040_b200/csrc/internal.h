@@ -213,7 +213,7 @@ cudaError_t launch_rollout_fused(const FusedLaunch& p, int32_t nodes, cudaStream
 constexpr size_t kTreeSmemLimit = 200 * 1024;   // per-node doubles beyond this live in node_scratch instead of shared memory
 struct FuseLaunch {
     const float* leaf_r; const float* logp; float* rbar; float* adv; int32_t* status;
-    double* node_scratch;      // [n_trees][2][nodes_cap], used when 16 bytes per node exceed kTreeSmemLimit
+    double* node_scratch;      // [n_trees][2][nodes_cap], used when three doubles per node exceed kTreeSmemLimit (trees of more than 8 533 nodes)
     LevelInfo lv; int32_t n_trees, nodes_cap, T, nodes; double beta_scaled; float eps, clip;
 };
 cudaError_t launch_fuse_advantage(const FuseLaunch& p, cudaStream_t s);
