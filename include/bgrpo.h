@@ -144,6 +144,19 @@ bgrpo_status bgrpo_velocity_linear_bind(bgrpo_tree* tree, const float* mu_dev, f
  * Errors: STATE (already at depth T; NULL v_dev without a bound velocity), CAPACITY (children exceed nodes_cap), CUDA. */
 bgrpo_status bgrpo_tree_step(bgrpo_tree* tree, int32_t split_flag, const float* v_dev, void* stream);
 
+/* tree_rollout: the remaining steps of the tree, depth .. T-1, in one host call (Algorithm 1, "Build rollout tree": for
+ * every step, the velocity of every live node, then the step that forks or advances it).  The same kernels in the same
+ * order as calling bgrpo_velocity_mlp (when packed_dev is given) and bgrpo_tree_step step by step, so every output is
+ * identical bit for bit; what it saves is the caller's per-call overhead, which on single-tree workloads (launches of
+ * 5-40 us) is comparable to the launches themselves.
+ *   split_flags_host  host array of T flags (indexed by step), non-zero = fork every node into K children
+ *   packed_dev        device, packed MLP weights (bgrpo_velocity_mlp_pack), or NULL for the bound linear velocity
+ *   v_dev             device [n_trees][W_max][D] float32 scratch for the velocities of the widest frontier (NULL allowed
+ *                     with packed_dev == NULL)
+ * Errors: those of the two calls (the tree keeps the depth it reached); INVALID_ARG, STATE as stated for them. */
+bgrpo_status bgrpo_tree_rollout(bgrpo_tree* tree, const uint8_t* split_flags_host, const void* packed_dev, int32_t hidden,
+                                float* v_dev, void* stream);
+
 /* tree_rollout_fused: all T steps of tree_step in one launch, for the bound closed-form velocity (Branch Rollout
  * Algorithm, where a prefix is computed once for all the leaves below it; Eq. 2; Algorithm 1 "Build rollout tree").
  * That velocity acts on every latent

@@ -65,6 +65,7 @@ _SIGNATURES = {
     "bgrpo_tree_reset": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p]),
     "bgrpo_velocity_linear_bind": (C.c_int, [C.c_void_p, C.c_void_p, C.c_float]),
     "bgrpo_tree_step": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "bgrpo_tree_rollout": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_rollout_fused": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "bgrpo_tree_logprob": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "bgrpo_velocity_mlp_packed_bytes": (C.c_size_t, [C.c_int32]),
@@ -171,6 +172,13 @@ def velocity_linear_bind(tree: Tree, mu, s0: float):
 
 def tree_step(tree: Tree, split_flag: int, v=None, stream=None):
     _check(lib.bgrpo_tree_step(tree.handle, int(split_flag), _ptr(v), _stream(stream)), "bgrpo_tree_step")
+
+
+def tree_rollout(tree: Tree, split_flags, packed=None, hidden: int = 0, v=None, stream=None):
+    """split_flags: a numpy uint8 array of T flags (kept by the caller) or any sequence."""
+    arr = split_flags if isinstance(split_flags, np.ndarray) and split_flags.dtype == np.uint8 else \
+        np.ascontiguousarray([1 if f else 0 for f in split_flags], dtype=np.uint8)
+    _check(lib.bgrpo_tree_rollout(tree.handle, arr.ctypes.data, _ptr(packed), hidden, _ptr(v), _stream(stream)), "bgrpo_tree_rollout")
 
 
 def tree_rollout_fused(tree: Tree, split_flags: Sequence[int], stream=None):

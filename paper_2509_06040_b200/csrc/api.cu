@@ -306,6 +306,22 @@ bgrpo_status bgrpo_tree_step(bgrpo_tree* t, int32_t split_flag, const float* v_d
     return BGRPO_OK;
 }
 
+bgrpo_status bgrpo_tree_rollout(bgrpo_tree* t, const uint8_t* split_flags_host, const void* packed_dev, int32_t hidden,
+                                float* v_dev, void* stream) {
+    if (!t || !split_flags_host) return fail(BGRPO_ERR_INVALID_ARG, "tree or split_flags is NULL");
+    if (packed_dev && !v_dev) return fail(BGRPO_ERR_INVALID_ARG, "the MLP velocity needs a velocity buffer");
+    if (!packed_dev && !t->mu) return fail(BGRPO_ERR_STATE, "no velocity: pass the packed MLP weights or bind a linear velocity");
+    for (int i = t->depth; i < t->desc.T; ++i) {
+        if (packed_dev) {
+            const bgrpo_status st = bgrpo_velocity_mlp(t, packed_dev, hidden, v_dev, stream);
+            if (st != BGRPO_OK) return st;
+        }
+        const bgrpo_status st = bgrpo_tree_step(t, split_flags_host[i] ? 1 : 0, packed_dev ? v_dev : nullptr, stream);
+        if (st != BGRPO_OK) return st;
+    }
+    return BGRPO_OK;
+}
+
 bgrpo_status bgrpo_tree_rollout_fused(bgrpo_tree* t, const uint8_t* split_flags_host, void* stream) {
     if (!t || !split_flags_host) return fail(BGRPO_ERR_INVALID_ARG, "tree or split_flags is NULL");
     if (t->depth != 0) return fail(BGRPO_ERR_STATE, "the whole-tree rollout starts from a freshly initialised or reset tree");

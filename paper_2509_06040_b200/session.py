@@ -46,6 +46,7 @@ class TreeSession:
         self.tree = None
         self.mu = self.target = self.packed = self.v = self.reward_draws = None
         self.pruned_steps = ()
+        self._split_flags = np.ascontiguousarray([1 if i in w.splits else 0 for i in range(w.T)], dtype=np.uint8)
 
     # -- inputs ---------------------------------------------------------------------------------------------------
     def upload_inputs(self, inp):
@@ -93,10 +94,11 @@ class TreeSession:
     def rollout(self, seed=None):
         self.init(seed)
         if self.fused_rollout:
-            B.tree_rollout_fused(self.tree, [1 if i in self.w.splits else 0 for i in range(self.w.T)])
-            return
-        for i in range(self.w.T):
-            self.step(i)
+            B.tree_rollout_fused(self.tree, self._split_flags)
+        elif self.w.velocity == "mlp":
+            B.tree_rollout(self.tree, self._split_flags, self.packed, self.w.hidden, self.v)       # T x [velocity, step], one host call
+        else:
+            B.tree_rollout(self.tree, self._split_flags)
 
     def rewards(self):
         w = self.w

@@ -185,6 +185,49 @@ def test_sharded_batch_draws_the_same_noise(B):
     assert torch.equal(whole.logp[2:], part.logp)
 
 
+def test_one_call_rollout_is_the_step_by_step_rollout(B):
+    """bgrpo_tree_rollout enqueues the same kernels as T x [velocity, tree_step] (Algorithm 1, "Build rollout tree"):
+    every output is identical bit for bit, for the closed-form and the MLP velocity, and it continues a tree that has
+    already taken some steps."""
+    for velocity, channels, hidden in (("linear", 4, 0), ("mlp", 64, 256)):
+        w = Workload(name="one_call", n_trees=2, tokens=150, channels=channels, T=5, K=3, splits=(0, 3), sigma=0.3,
+                     velocity=velocity, reward="mixture", hidden=hidden or 3072, branch_corr_s=2.0)
+        inp = make_inputs(w)
+        a, b, c = _session(w), _session(w), _session(w)
+        for s in (a, b, c):
+            s.upload_inputs(inp)
+            s.init()
+        flags = [1 if i in w.splits else 0 for i in range(w.T)]
+        for i in range(w.T):                                   # a: one call per step
+            a.step(i)
+        if velocity == "mlp":                                  # b: one call for the tree; c: two steps, then the rest
+            B.tree_rollout(b.tree, flags, b.packed, w.hidden, b.v)
+            c.step(0); c.step(1)
+            B.tree_rollout(c.tree, flags, c.packed, w.hidden, c.v)
+        else:
+            B.tree_rollout(b.tree, flags)
+            c.step(0); c.step(1)
+            B.tree_rollout(c.tree, flags)
+        torch.cuda.synchronize()
+        for s in (a, b, c):
+            B.tree_sync_status(s.tree)
+        for other in (b, c):
+            assert B.tree_stats(other.tree) == B.tree_stats(a.tree)
+            assert torch.equal(a.latents, other.latents) and torch.equal(a.logp[:, :w.nodes], other.logp[:, :w.nodes])
+            assert torch.equal(a.node_table, other.node_table)
+        with pytest.raises(B.BgrpoError) as e:                 # the tree is complete: nothing left to do is fine, a step is not
+            B.tree_step(b.tree, 0, b.v if velocity == "mlp" else None)
+        assert e.value.status == B.ERR_STATE
+        B.tree_rollout(b.tree, flags, b.packed if velocity == "mlp" else None, w.hidden if velocity == "mlp" else 0, b.v)
+    wl = Workload(name="one_call_err", n_trees=1, tokens=16, channels=4, T=2, K=2, splits=(0,), sigma=0.3, velocity="linear",
+                  reward="neg_mse_mu")
+    s = _session(wl)
+    s.init()                                                    # no velocity bound, no weights given
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_rollout(s.tree, [1, 0])
+    assert e.value.status == B.ERR_STATE
+
+
 # ---------------------------------------------------------------------------------------------- given velocity (MLP stand-in path)
 def test_step_with_supplied_velocity_and_logprob_recompute(B):
     """tree_step with a velocity buffer (the MLP configurations' path), teacher-forced: the oracle's MLP
