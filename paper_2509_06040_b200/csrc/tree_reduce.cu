@@ -60,6 +60,16 @@ fuse_advantage_kernel(const FuseLaunch p) {
                 ls[off + j] = (la ? la[c0] : beta * static_cast<double>(p.logp[row0 + c0])) + ls[c0];
                 continue;
             }
+            if (beta == 0.0) {   // uniform weights: every child of a node has the same number of leaves below it, so the
+                                 // leaf mean of the parent is the plain mean of its children's leaf means
+                double R = 0.0;
+#pragma unroll
+                for (int b = 0; b < BGRPO_MAX_K; ++b)
+                    if (b < fan) R += rb[c0 + b];
+                rb[off + j] = R / fan;
+                ls[off + j] = 0.0;
+                continue;
+            }
             double a[BGRPO_MAX_K];
             double m = -INFINITY;
 #pragma unroll
