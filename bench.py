@@ -51,7 +51,7 @@ NCU_TRAFFIC = {
                            "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d569995ada83"},
     "step_kernel_mlp": {"bytes": 531.169024e6 + 215.974400e6, "units": 32 * 16 * 129600,         # profiles/step_kernel_image_batch.md
                         "sources": ("tree_step.cu", "philox.cuh"), "shape": "kStep", "source_hash": "d569995ada83"},
-    "mlp_velocity_kernel": {"bytes": 266.334720e6 + 215.852032e6, "units": 1036800,       # profiles/mlp_velocity_kernel_image_batch.md
+    "mlp_velocity_kernel": {"bytes": 266.295296e6 + 213.379328e6, "units": 1036800,       # profiles/mlp_velocity_kernel_image_batch.md
                             "sources": ("mlp_velocity.cu",), "shape": "kMlp", "source_hash": "74593cdd150d"},
     "rollout_fused_kernel": {"bytes": 16.816640e6 + 866.172416e6, "units": 110 * 2096640,  # profiles/rollout_fused_kernel_video.md
                              "sources": ("tree_fused.cu", "philox.cuh"), "shape": "kFused", "source_hash": "d4f0707c5632"},
