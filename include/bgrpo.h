@@ -258,6 +258,20 @@ bgrpo_status bgrpo_tree_levels(const bgrpo_tree* tree, int32_t n, int32_t* width
  * BGRPO_ERR_CAPACITY (a device-side index check failed; the access was skipped).  The word is cleared afterwards. */
 bgrpo_status bgrpo_tree_sync_status(bgrpo_tree* tree, void* stream);
 
+/* Saving and restoring a tree (no counterpart in the paper's method; its training loop checkpoints every 40 steps,
+ * hyper-parameter table).  A tree's state is the caller's device buffers plus a small host record: description, t-grid,
+ * level layout, hybrid-schedule flags, depth.  bgrpo_tree_export first enqueues the kernel that completes any pending
+ * log-prob sums (so buffers.logp is final once `stream` has run), then writes the record to blob_host
+ * (bgrpo_tree_export_bytes() bytes).  bgrpo_tree_import builds a new handle from such a record and a set of buffers that
+ * hold what the exported tree's buffers held (the same allocations, or copies made after `stream` had run; scratch may be
+ * fresh), without launching a kernel; it clears the status word and the MLP stage's tickets on `stream`.  A bound linear
+ * velocity is a device pointer and is not saved: call bgrpo_velocity_linear_bind again.  Continuing an imported tree gives
+ * the bits an uninterrupted tree gives.  Errors: INVALID_ARG (NULL, foreign or inconsistent record, misaligned buffer),
+ * CAPACITY (blob or scratch too small), CUDA. */
+size_t       bgrpo_tree_export_bytes(void);
+bgrpo_status bgrpo_tree_export(bgrpo_tree* tree, void* blob_host, size_t blob_bytes, void* stream);
+bgrpo_status bgrpo_tree_import(const void* blob_host, size_t blob_bytes, const bgrpo_buffers* buffers, void* stream, bgrpo_tree** out);
+
 /* Debug build with device-side index checks (library compiled with -DBGRPO_DEBUG_BOUNDS; no counterpart in the paper).
  * In that build every kernel tests the row, chunk and element indices it derives against the extents it was launched
  * with; a failed test sets a bit of the status word and the access is skipped - nothing traps - and

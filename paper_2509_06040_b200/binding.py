@@ -86,6 +86,9 @@ _SIGNATURES = {
     "bgrpo_philox_words_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
     "bgrpo_philox_normal_fill": (C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_int64, C.c_void_p]),
     "bgrpo_reward_mse_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p]),
+    "bgrpo_tree_export_bytes": (C.c_size_t, []),
+    "bgrpo_tree_export": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "bgrpo_tree_import": (C.c_int, [C.c_void_p, C.c_size_t, C.POINTER(Buffers), C.c_void_p, C.POINTER(C.c_void_p)]),
     "bgrpo_debug_bounds": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "bgrpo_tree_destroy": (None, [C.c_void_p]),
     "bgrpo_status_string": (C.c_char_p, [C.c_int]),
@@ -272,6 +275,20 @@ def tree_levels(tree: Tree):
 
 def tree_sync_status(tree: Tree, stream=None):
     _check(lib.bgrpo_tree_sync_status(tree.handle, _stream(stream)), "bgrpo_tree_sync_status")
+
+
+def tree_export(tree: Tree, stream=None) -> bytes:
+    buf = C.create_string_buffer(lib.bgrpo_tree_export_bytes())
+    _check(lib.bgrpo_tree_export(tree.handle, buf, len(buf), _stream(stream)), "bgrpo_tree_export")
+    return buf.raw
+
+
+def tree_import(blob: bytes, latents, node_table, logp, rbar, adv, mask, scratch, stream=None, keep=()) -> Tree:
+    b = Buffers(_ptr(latents), _ptr(node_table), _ptr(logp), _ptr(rbar), _ptr(adv), _ptr(mask), _ptr(scratch),
+                scratch.numel() * scratch.element_size())
+    h = C.c_void_p()
+    _check(lib.bgrpo_tree_import(blob, len(blob), C.byref(b), _stream(stream), C.byref(h)), "bgrpo_tree_import")
+    return Tree(h.value, None, (latents, node_table, logp, rbar, adv, mask, scratch) + tuple(keep))
 
 
 def debug_bounds(tree: Optional[Tree], trip: bool = False, stream=None):

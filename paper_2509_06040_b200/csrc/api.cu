@@ -81,6 +81,44 @@ void fill_coefficients(bgrpo_tree* t) {
     }
 }
 
+// Everything of the handle that follows from the description and the buffers alone: sizes, noise mixing, the carving of
+// the scratch allocation.  No velocity bound, every step stochastic, nothing pending.
+void bind_buffers(bgrpo_tree* t, const bgrpo_buffers* b) {
+    const bgrpo_tree_desc* desc = &t->desc;
+    t->buf = *b;
+    t->D = static_cast<int64_t>(desc->tokens) * desc->channels;
+    t->nchunks = nchunks_of(t->D);
+    t->nchunks_step = nchunks_step_of(t->D);
+    t->nchunks_reward = static_cast<int32_t>((t->D / 4 + kRewardChunkVec - 1) / kRewardChunkVec);
+    t->independent = !(std::isfinite(desc->branch_corr_s) && desc->branch_corr_s >= 0.0f);
+    if (t->independent) {
+        t->mix_shared = 0.0f;
+        t->mix_innov = 1.0f;
+    } else {
+        const double s = desc->branch_corr_s, n = std::sqrt(1.0 + s * s);
+        t->mix_shared = static_cast<float>(1.0 / n);
+        t->mix_innov = static_cast<float>(s / n);
+    }
+    t->mu = nullptr;
+    t->s0 = 0.0f;
+    t->ode_bits = 0;
+    char* sc = static_cast<char*>(b->scratch);
+    const size_t rows = static_cast<size_t>(desc->n_trees) * desc->nodes_cap;
+    t->status = reinterpret_cast<int32_t*>(sc);
+    t->counters = reinterpret_cast<unsigned int*>(sc + kScratchHeader);
+    t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
+    t->node_scratch = t->partials + rows * static_cast<size_t>(t->nchunks) * 3;
+    t->partialsf = reinterpret_cast<float*>(t->node_scratch + rows * 2);
+    t->mlp_tickets = nullptr;
+    t->mlp_partials = nullptr;
+    if (desc->channels == BGRPO_MLP_CHANNELS) {
+        const size_t used = reinterpret_cast<char*>(t->partialsf + rows * static_cast<size_t>(partials_per_row(t->D))) - sc;
+        t->mlp_tickets = reinterpret_cast<unsigned int*>(sc + ((used + 255) / 256) * 256);
+        t->mlp_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(t->mlp_tickets) + kMlpTicketBytes);
+    }
+    t->pending.logp_out = nullptr;
+}
+
 bool tree_complete(const bgrpo_tree* t) { return t->depth == t->desc.T; }
 
 // Enqueues the small kernel that adds up a level's pending log-prob partials, if there are any.
@@ -168,40 +206,9 @@ bgrpo_status bgrpo_tree_init(const bgrpo_tree_desc* desc, const bgrpo_buffers* b
     bgrpo_tree* t = new (std::nothrow) bgrpo_tree();
     if (!t) return fail(BGRPO_ERR_INVALID_ARG, "out of host memory");
     t->desc = *desc;
-    t->buf = *b;
     std::memcpy(t->t_grid, desc->t_grid, sizeof(float) * (desc->T + 1));
     t->desc.t_grid = t->t_grid;
-    t->D = static_cast<int64_t>(desc->tokens) * desc->channels;
-    t->nchunks = nchunks_of(t->D);
-    t->nchunks_step = nchunks_step_of(t->D);
-    t->nchunks_reward = static_cast<int32_t>((t->D / 4 + kRewardChunkVec - 1) / kRewardChunkVec);
-    t->independent = !(std::isfinite(desc->branch_corr_s) && desc->branch_corr_s >= 0.0f);
-    if (t->independent) {
-        t->mix_shared = 0.0f;
-        t->mix_innov = 1.0f;
-    } else {
-        const double s = desc->branch_corr_s, n = std::sqrt(1.0 + s * s);
-        t->mix_shared = static_cast<float>(1.0 / n);
-        t->mix_innov = static_cast<float>(s / n);
-    }
-    t->mu = nullptr;
-    t->s0 = 0.0f;
-    t->ode_bits = 0;
-    char* sc = static_cast<char*>(b->scratch);
-    const size_t rows = static_cast<size_t>(desc->n_trees) * desc->nodes_cap;
-    t->status = reinterpret_cast<int32_t*>(sc);
-    t->counters = reinterpret_cast<unsigned int*>(sc + kScratchHeader);
-    t->partials = reinterpret_cast<double*>(sc + kScratchHeader + ((rows * sizeof(unsigned int) + 255) / 256) * 256);
-    t->node_scratch = t->partials + rows * static_cast<size_t>(t->nchunks) * 3;
-    t->partialsf = reinterpret_cast<float*>(t->node_scratch + rows * 2);
-    t->mlp_tickets = nullptr;
-    t->mlp_partials = nullptr;
-    if (desc->channels == BGRPO_MLP_CHANNELS) {
-        const size_t used = reinterpret_cast<char*>(t->partialsf + rows * static_cast<size_t>(partials_per_row(t->D))) - sc;
-        t->mlp_tickets = reinterpret_cast<unsigned int*>(sc + ((used + 255) / 256) * 256);
-        t->mlp_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(t->mlp_tickets) + kMlpTicketBytes);
-    }
-    t->pending.logp_out = nullptr;
+    bind_buffers(t, b);
     fill_coefficients(t);
     st = bgrpo_tree_reset(t, desc->seed, stream);
     if (st == BGRPO_OK && t->mlp_tickets) {      // the MLP stage's tile tickets start at zero and return to zero after every launch
@@ -656,6 +663,77 @@ bgrpo_status bgrpo_velocity_mlp(bgrpo_tree* t, const void* packed_dev, int32_t h
                                t->desc.n_trees, static_cast<int64_t>(t->lv.width[i]) * t->desc.tokens, packed_dev, hidden,
                                v_out_dev, t->mlp_partials, t->mlp_tickets, t->status, as_stream(stream));
     return e == cudaSuccess ? BGRPO_OK : cuda_fail(e, "mlp kernel");
+}
+
+namespace {
+// Host state of a tree as it is saved: everything bgrpo_tree_import needs besides the device buffers themselves.
+struct TreeBlob {
+    uint32_t magic, version;
+    bgrpo_tree_desc desc;                // t_grid pointer not meaningful outside the process: the values follow
+    float t_grid[BGRPO_MAX_T + 1];
+    LevelInfo lv;
+    uint64_t ode_bits;
+    int32_t depth;
+    float s0;                            // 0: no linear velocity was bound
+};
+constexpr uint32_t kBlobMagic = 0x42475250u, kBlobVersion = 1u;      // "BGRP"
+}  // namespace
+
+size_t bgrpo_tree_export_bytes(void) { return sizeof(TreeBlob); }
+
+bgrpo_status bgrpo_tree_export(bgrpo_tree* t, void* blob_host, size_t blob_bytes, void* stream) {
+    if (!t || !blob_host) return fail(BGRPO_ERR_INVALID_ARG, "tree or blob is NULL");
+    if (blob_bytes < sizeof(TreeBlob)) return fail(BGRPO_ERR_CAPACITY, "blob smaller than bgrpo_tree_export_bytes()");
+    const cudaError_t e = flush_pending(t, as_stream(stream));     // the last level's log-probs become final in buffers.logp
+    if (e != cudaSuccess) return cuda_fail(e, "log-prob flush kernel");
+    TreeBlob b;
+    std::memset(&b, 0, sizeof(b));
+    b.magic = kBlobMagic;
+    b.version = kBlobVersion;
+    b.desc = t->desc;
+    b.desc.t_grid = nullptr;
+    std::memcpy(b.t_grid, t->t_grid, sizeof(b.t_grid));
+    b.lv = t->lv;
+    b.ode_bits = t->ode_bits;
+    b.depth = t->depth;
+    b.s0 = t->mu ? t->s0 : 0.0f;
+    std::memcpy(blob_host, &b, sizeof(b));
+    return BGRPO_OK;
+}
+
+bgrpo_status bgrpo_tree_import(const void* blob_host, size_t blob_bytes, const bgrpo_buffers* buffers, void* stream, bgrpo_tree** out) {
+    if (!blob_host || !buffers || !out) return fail(BGRPO_ERR_INVALID_ARG, "blob, buffers or out is NULL");
+    if (blob_bytes < sizeof(TreeBlob)) return fail(BGRPO_ERR_INVALID_ARG, "blob too small");
+    TreeBlob b;
+    std::memcpy(&b, blob_host, sizeof(b));
+    if (b.magic != kBlobMagic || b.version != kBlobVersion) return fail(BGRPO_ERR_INVALID_ARG, "not a tree blob of this library version");
+    b.desc.t_grid = b.t_grid;
+    bgrpo_status st = check_desc(&b.desc);
+    if (st != BGRPO_OK) return st;
+    if (b.depth < 0 || b.depth > b.desc.T || b.lv.offset[b.depth + 1] > b.desc.nodes_cap) return fail(BGRPO_ERR_INVALID_ARG, "blob describes a tree that does not fit its own description");
+    if (!buffers->latents || !buffers->node_table || !buffers->logp || !buffers->rbar || !buffers->adv || !buffers->mask || !buffers->scratch)
+        return fail(BGRPO_ERR_INVALID_ARG, "a device buffer is NULL");
+    if (!aligned(buffers->latents, 16) || !aligned(buffers->scratch, 256)) return fail(BGRPO_ERR_INVALID_ARG, "misaligned device buffer");
+    if (buffers->scratch_bytes < scratch_bytes_of(&b.desc)) return fail(BGRPO_ERR_CAPACITY, "scratch_bytes too small");
+    bgrpo_tree* t = new (std::nothrow) bgrpo_tree();
+    if (!t) return fail(BGRPO_ERR_INVALID_ARG, "out of host memory");
+    t->desc = b.desc;
+    std::memcpy(t->t_grid, b.t_grid, sizeof(t->t_grid));
+    t->desc.t_grid = t->t_grid;
+    bind_buffers(t, buffers);
+    t->lv = b.lv;
+    t->ode_bits = b.ode_bits;
+    t->depth = b.depth;
+    fill_coefficients(t);
+    // the status word and the MLP tile tickets live in scratch, which may be a fresh allocation: both start at zero
+    cudaError_t e = cudaMemsetAsync(t->status, 0, sizeof(int32_t), as_stream(stream));
+    if (e == cudaSuccess && t->mlp_tickets) e = cudaMemsetAsync(t->mlp_tickets, 0, kMlpTicketBytes, as_stream(stream));
+    if (e != cudaSuccess) {
+        delete t;
+        return cuda_fail(e, "clearing the status word and the MLP tickets");
+    }
+    *out = t;
+    return BGRPO_OK;
 }
 
 bgrpo_status bgrpo_debug_bounds(bgrpo_tree* t, int32_t trip, void* stream) {

@@ -228,6 +228,56 @@ def test_one_call_rollout_is_the_step_by_step_rollout(B):
     assert e.value.status == B.ERR_STATE
 
 
+def test_export_import_continues_bit_identically(B):
+    """A tree is saved after two steps (its host record plus copies of its device buffers, scratch left behind), restored
+    into a new handle over the copies, and continued: every output equals the uninterrupted tree's bit for bit - for the
+    closed-form velocity with the hybrid ODE-SDE schedule and for the MLP velocity."""
+    for velocity, channels in (("linear", 4), ("mlp", 64)):
+        w = Workload(name="resume", n_trees=2, tokens=150, channels=channels, T=5, K=2, splits=(0, 3), sigma=0.3,
+                     velocity=velocity, reward="neg_mse_target", hidden=256, branch_corr_s=2.0, width_mode=B.WIDTH_PER_SPLIT_TOPK, width_k=1)
+        inp = make_inputs(w)
+        sde = [1, 0, 1, 1, 1]
+        whole, first = _session(w, nodes_cap=w.nodes + 2), _session(w, nodes_cap=w.nodes + 2)
+        for s in (whole, first):
+            s.upload_inputs(inp)
+            s.init()
+            B.tree_set_sde_steps(s.tree, sde)
+        for i in range(w.T):
+            whole.step(i)
+        first.step(0)
+        first.step(1)
+        blob = B.tree_export(first.tree)
+        assert len(blob) == B.lib.bgrpo_tree_export_bytes()
+        torch.cuda.synchronize()
+        # the restored tree lives in copies of the buffers; its scratch is a fresh allocation
+        second = _session(w, nodes_cap=w.nodes + 2)
+        second.upload_inputs(inp)
+        for name in ("latents", "node_table", "logp"):
+            getattr(second, name).copy_(getattr(first, name))
+        second.scratch.fill_(0xAB)
+        second.tree = B.tree_import(blob, second.latents, second.node_table, second.logp, second.rbar, second.adv, second.mask, second.scratch)
+        if velocity == "linear":
+            B.velocity_linear_bind(second.tree, second.mu, f32(w.s0))
+        assert B.tree_stats(second.tree) == B.tree_stats(first.tree)
+        for i in range(2, w.T):
+            second.step(i)
+        for s in (whole, second):
+            s.rewards(); s.fuse_advantage(); s.prune()
+        torch.cuda.synchronize()
+        B.tree_sync_status(second.tree)
+        n = w.nodes
+        assert torch.equal(whole.latents[:, :n], second.latents[:, :n])
+        assert torch.equal(whole.logp[:, :n], second.logp[:, :n])
+        cap = whole.nodes_cap
+        assert torch.equal(whole.node_table.view(4, w.n_trees, cap)[:, :, :n], second.node_table.view(4, w.n_trees, cap)[:, :, :n])
+        assert torch.equal(whole.leaf_r, second.leaf_r) and torch.equal(whole.adv[:, :n], second.adv[:, :n])
+        assert torch.equal(whole.mask[:, :n], second.mask[:, :n])
+    # a foreign record is refused
+    with pytest.raises(B.BgrpoError) as e:
+        B.tree_import(b"\0" * len(blob), second.latents, second.node_table, second.logp, second.rbar, second.adv, second.mask, second.scratch)
+    assert e.value.status == B.ERR_INVALID_ARG
+
+
 # ---------------------------------------------------------------------------------------------- given velocity (MLP stand-in path)
 def test_step_with_supplied_velocity_and_logprob_recompute(B):
     """tree_step with a velocity buffer (the MLP configurations' path), teacher-forced: the oracle's MLP
