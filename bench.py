@@ -260,6 +260,7 @@ def oracle_pass(w, fraction, workers):
     topo = otree.build_topology(w.T, w.K, w.splits)
     unit = 4 if w.velocity == "linear" else w.channels
     total_units = w.D // unit
+    workers = max(1, min(workers, total_units))          # never more processes than slices of the row
     n_units = min(total_units, max(workers, int(total_units * fraction)))
     bounds = np.linspace(0, n_units, workers + 1).astype(int)
     jobs = [(w.name, int(bounds[k]) * unit, int(bounds[k + 1] - bounds[k]) * unit) for k in range(workers)]
@@ -317,6 +318,7 @@ def cpu_baseline(w, single=True):
     workers = min(nproc, 64)
     f1, fn = ORACLE_SAMPLE.get(w.name, (0.02, 0.1))
     out = {"unit": UNIT, "kind": "oracle", "nproc": nproc}
+    workers = max(1, min(workers, w.D // (4 if w.velocity == "linear" else w.channels)))
     dt_n, v_n, desc_n = oracle_pass(w, fn, workers)
     out.update({"value": r4(v_n), "cores": workers, "sample": desc_n, "sample_seconds": r4(dt_n)})
     if single:
