@@ -90,3 +90,19 @@ def test_depth_window_matches_the_stated_schedule(B):
 def test_mlp_packed_bytes(B):
     assert B.velocity_mlp_packed_bytes(3072) >= 2 * 64 * 3072 * 2
     assert B.velocity_mlp_packed_bytes(100) == 0
+
+
+def test_binding_refuses_to_import_without_the_library(tmp_path):
+    """There is no CPU or PyTorch fallback: a copy of the package without libbgrpo.so fails at import, loudly."""
+    import shutil
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_2509_06040_b200"
+    pkg.mkdir()
+    src = os.path.join(ROOT, "paper_2509_06040_b200")
+    for name in ("__init__.py", "binding.py", "session.py"):
+        shutil.copy(os.path.join(src, name), pkg / name)
+    out = subprocess.run([sys.executable, "-c", "import paper_2509_06040_b200.binding"], cwd=tmp_path, capture_output=True, text=True,
+                         env={k: v for k, v in os.environ.items() if k != "PYTHONPATH"})
+    assert out.returncode != 0
+    assert "libbgrpo.so is missing" in out.stderr and "no CPU or PyTorch fallback" in out.stderr
